@@ -1,0 +1,144 @@
+"""TEST INFRASTRUCTURE -- not part of the product path.
+
+ctypes front end of the CPU oracle (``cg_oracle.cpp``): the fused GEMM + epilogue
+``D = act(alpha*A@B + bias) + beta*R`` in single-threaded fp64.  Only tests, the smoke check
+and the benchmark's CPU-baseline leg may import this module; the CUDA package never does.
+
+All matrices travel as numpy arrays: bf16 operands as ``uint16`` bit patterns, the bias as
+``float32`` (or ``uint16`` bf16 bits together with ``FLAG_BIAS_BF16``).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+ACT_NONE, ACT_RELU, ACT_GELU_TANH, ACT_SILU = 0, 1, 2, 3
+FLAG_B_COLMAJOR = 1 << 8
+FLAG_BIAS_BF16 = 1 << 9
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "cg_oracle.cpp")
+_lib = None
+
+
+def _host_tag() -> str:
+    """Short hash of this host's CPU model and ISA flags: -march=native code built on one
+    machine must not be loaded on another, so the library file name carries the tag."""
+    import hashlib
+    text = ""
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.startswith(("model name", "flags")):
+                    text += line
+                if line.strip() == "" and text:
+                    break
+    except OSError:
+        pass
+    return hashlib.sha1(text.encode()).hexdigest()[:10]
+
+
+_LIB = os.path.join(_HERE, f"libcg_oracle.{_host_tag()}.so")
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ (no fused multiply-add, no fast-math); returns the .so path."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["g++", "-O3", "-march=native", "-std=c++17", "-ffp-contract=off", "-fno-fast-math",
+               "-fPIC", "-shared", "-o", _LIB, _SRC]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        vp, i64, dbl, ci = ctypes.c_void_p, ctypes.c_int64, ctypes.c_double, ctypes.c_int
+        lib.cg_ref_gemm_epilogue.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, i64, dbl, dbl, ci]
+        lib.cg_ref_gemm_epilogue.restype = ci
+        for name in ("cg_ref_gemm_epilogue_rows", "cg_ref_gemm_epilogue_points"):
+            fn = getattr(lib, name)
+            fn.argtypes = [vp, vp, vp, vp, vp, i64, vp, vp, i64, i64, i64, i64, dbl, dbl, ci]
+            fn.restype = ci
+        lib.cg_ref_activation.argtypes = [ci, dbl]
+        lib.cg_ref_activation.restype = dbl
+        lib.cg_ref_f64_to_bf16.argtypes = [dbl]
+        lib.cg_ref_f64_to_bf16.restype = ctypes.c_uint16
+        lib.cg_ref_bf16_to_f64.argtypes = [ctypes.c_uint16]
+        lib.cg_ref_bf16_to_f64.restype = dbl
+        _lib = lib
+    return _lib
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _check(A, B, bias, R, M, N, K, batch, act):
+    for name, x in (("A", A), ("B", B)):
+        if x.dtype != np.uint16 or not x.flags.c_contiguous:
+            raise TypeError(f"{name} must be a C-contiguous uint16 (bf16 bits) array")
+    if A.size != batch * M * K or B.size != batch * K * N:
+        raise ValueError("operand sizes do not match M, N, K, batch")
+    if bias is not None:
+        want = np.uint16 if act & FLAG_BIAS_BF16 else np.float32
+        if bias.dtype != want or bias.size != N or not bias.flags.c_contiguous:
+            raise TypeError("bias must be a contiguous length-N array of the flagged dtype")
+    if R is not None and (R.dtype != np.uint16 or R.size != batch * M * N or not R.flags.c_contiguous):
+        raise TypeError("R must be a C-contiguous uint16 array of batch*M*N elements")
+
+
+def gemm_epilogue(A, B, bias, R, M, N, K, batch, alpha, beta, act, want_bf16=True):
+    """Whole problem.  Returns (D64 [batch,M,N] float64, Dbf16 bits [batch,M,N] uint16 or None)."""
+    _check(A, B, bias, R, M, N, K, batch, act)
+    d64 = np.empty((batch, M, N), dtype=np.float64)
+    d16 = np.empty((batch, M, N), dtype=np.uint16) if want_bf16 else None
+    rc = _load().cg_ref_gemm_epilogue(_ptr(A), _ptr(B), _ptr(bias), _ptr(R), _ptr(d64), _ptr(d16),
+                                      M, N, K, batch, float(alpha), float(beta), int(act))
+    if rc != 0:
+        raise ValueError("oracle rejected the arguments")
+    return d64, d16
+
+
+def gemm_epilogue_rows(A, B, bias, R, rows, M, N, K, batch, alpha, beta, act):
+    """Rows ``rows[i] = b*M + m`` only.  Returns (D64 [len(rows),N], Dbf16 bits [len(rows),N])."""
+    _check(A, B, bias, R, M, N, K, batch, act)
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    d64 = np.empty((rows.size, N), dtype=np.float64)
+    d16 = np.empty((rows.size, N), dtype=np.uint16)
+    rc = _load().cg_ref_gemm_epilogue_rows(_ptr(A), _ptr(B), _ptr(bias), _ptr(R), _ptr(rows), rows.size,
+                                           _ptr(d64), _ptr(d16), M, N, K, batch, float(alpha),
+                                           float(beta), int(act))
+    if rc != 0:
+        raise ValueError("oracle rejected the arguments")
+    return d64, d16
+
+
+def gemm_epilogue_points(A, B, bias, R, idx, M, N, K, batch, alpha, beta, act):
+    """Single outputs at flat indices ``(b*M + m)*N + n``.  Returns (D64 [len(idx)], bf16 bits)."""
+    _check(A, B, bias, R, M, N, K, batch, act)
+    idx = np.ascontiguousarray(idx, dtype=np.int64)
+    d64 = np.empty(idx.size, dtype=np.float64)
+    d16 = np.empty(idx.size, dtype=np.uint16)
+    rc = _load().cg_ref_gemm_epilogue_points(_ptr(A), _ptr(B), _ptr(bias), _ptr(R), _ptr(idx), idx.size,
+                                             _ptr(d64), _ptr(d16), M, N, K, batch, float(alpha),
+                                             float(beta), int(act))
+    if rc != 0:
+        raise ValueError("oracle rejected the arguments")
+    return d64, d16
+
+
+def activation(act, t):
+    return _load().cg_ref_activation(int(act), float(t))
+
+
+def f64_to_bf16(v):
+    return int(_load().cg_ref_f64_to_bf16(float(v)))
+
+
+def bf16_to_f64(h):
+    return float(_load().cg_ref_bf16_to_f64(int(h)))
