@@ -1,0 +1,137 @@
+/*
+ * cg -- fused bf16 GEMM + epilogue for NVIDIA B200 (sm_100a), C ABI.
+ *
+ *     D[b,m,n] = act( alpha * sum_k A[b,m,k] * B[b,k,n] + bias[n] ) + beta * R[b,m,n]
+ *
+ * bf16 operands, fp32 accumulation in tensor memory, bf16 output, one kernel launch per call.
+ * This is the kernel family the paper's optimisation prompts describe for GEMM-like work:
+ * CTA tiling, tensor-core MMA, swizzled shared-memory operand layout, multi-stage asynchronous
+ * loads, split-K (Level-1 optimisation prompt, GEMM section, items 1-9) with bias / scale /
+ * add / activation fused into the producer's write-back so that the output is written once
+ * and no intermediate tensor exists (Level-2 optimisation prompt, "SECOND PRIORITY: FUSION",
+ * item 1; GEMM strategy "prefer epilogue fusion first").  The alpha/beta convention is the one
+ * of the paper's square-GEMM listing (C = alpha*Acc + beta*C).  The task formulation in the
+ * Method section (replace the reference computation by one custom-kernel call behind the same
+ * interface, no library fallback) is the model for this boundary.
+ *
+ * Conventions for every function:
+ *   - the return value is a cg status code; nothing throws;
+ *   - on any error nothing is enqueued and D is not touched;
+ *   - device pointers are plain CUDA device addresses owned by the caller; they must stay
+ *     valid until the stream has run the call; the handle owns only its workspace;
+ *   - calls on one handle are serialised by a mutex; use one handle per concurrent stream.
+ */
+#ifndef CG_H_
+#define CG_H_
+
+#include <stddef.h>
+
+#if defined(__GNUC__)
+#define CG_API __attribute__((visibility("default")))
+#else
+#define CG_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct cg_context* cg_handle_t;
+
+enum {
+  CG_OK = 0,
+  CG_ERR_INVALID_ARG = 1, /* NULL operand, non-positive size, unknown activation, R missing with beta != 0 */
+  CG_ERR_UNSUPPORTED = 2, /* N or K not a multiple of 8, a pointer not 16-byte aligned, size beyond limits */
+  CG_ERR_ARCH = 3,        /* the device is not compute capability 10.0 */
+  CG_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed; see cg_last_error */
+  CG_ERR_WORKSPACE = 5,   /* a forced split plan does not fit the handle's workspace */
+  CG_ERR_TIMEOUT = 6      /* device side: a bounded wait inside the kernel expired (reported by cg_last_error) */
+};
+
+/* Low byte of `act`. */
+enum { CG_ACT_NONE = 0, CG_ACT_RELU = 1, CG_ACT_GELU_TANH = 2, CG_ACT_SILU = 3 };
+/* OR-ed into `act`: operand layout / dtype that the argument list has no slot for. */
+enum {
+  CG_FLAG_B_COLMAJOR = 1 << 8, /* B is stored [batch,N,K] (element (k,n) at n*K + k) */
+  CG_FLAG_BIAS_BF16 = 1 << 9   /* bias is bf16 instead of fp32 */
+};
+
+/*
+ * Creates a handle on CUDA device `device` (made current for the call).  `workspace_bytes`
+ * is the size of the device scratch used by split-K / stream-K plans (fp32 partial tiles and
+ * per-tile ticket counters); 0 selects the default of 64 MiB.  Allocates device memory.
+ */
+CG_API int cg_create(cg_handle_t* out, int device, size_t workspace_bytes);
+
+/*
+ * Enqueues one fused GEMM + epilogue on `stream` (a cudaStream_t passed as void*; NULL is the
+ * legacy default stream).  Asynchronous: never synchronises.
+ *
+ *   A     device, bf16 [batch,M,K] row-major, dense, 16-byte aligned
+ *   B     device, bf16 [batch,K,N] row-major; with CG_FLAG_B_COLMAJOR bf16 [batch,N,K]
+ *   bias  device, fp32 [N] (bf16 [N] with CG_FLAG_BIAS_BF16), shared by all rows and batch
+ *         entries, not scaled by alpha; NULL means zero
+ *   R     device, bf16 [batch,M,N] row-major; read only when beta != 0 (may be NULL otherwise);
+ *         may alias D exactly (in-place residual)
+ *   D     device, bf16 [batch,M,N] row-major, written once, never read; must not overlap A or B
+ *   M,N,K,batch >= 1; N % 8 == 0 and K % 8 == 0 (16-byte row pitch for the tensor maps)
+ *   act   activation in the low byte, CG_FLAG_* above it
+ *
+ * Accumulation is fp32 (tensor cores), the epilogue is fp32, the store rounds to nearest even.
+ * The activation is applied to alpha*A*B + bias; beta*R is added after it.
+ */
+CG_API int cg_gemm_epilogue(cg_handle_t h, const void* A, const void* B, const void* bias, const void* R, void* D,
+                     int M, int N, int K, int batch, float alpha, float beta, int act, void* stream);
+
+/*
+ * Same operation with HOST buffers (same shapes, dtypes and layouts as above, in host memory;
+ * pinned memory makes the copies asynchronous and faster).  Copies the operands to device
+ * staging buffers owned by the handle (grown on demand and kept), runs the kernel, copies D
+ * back and synchronises `stream` before returning.  The end-to-end path of the benchmark.
+ */
+CG_API int cg_gemm_epilogue_host(cg_handle_t h, const void* A, const void* B, const void* bias, const void* R,
+                          void* D, int M, int N, int K, int batch, float alpha, float beta, int act,
+                          void* stream);
+
+/*
+ * Plan override for tests and benchmarking; all-zero (the default) lets the heuristic choose.
+ * A non-zero field forces that choice for the following calls on this handle.
+ */
+typedef struct cg_tuning {
+  int tile_n;    /* 64, 128 or 256: accumulator tile width                                  */
+  int cta_group; /* 1 = one CTA per 128-row tile, 2 = CTA pair sharing a 256-row tile       */
+  int num_units; /* number of contiguous k-block ranges the iteration space is cut into:
+                    = number of tiles -> data-parallel, a multiple of it -> split-K,
+                    anything else -> stream-K (cta_group 1 only)                            */
+  int stages;    /* depth of the shared-memory operand ring (clamped to what fits)          */
+  int group_m;   /* raster: m-tiles walked before stepping to the next n-tile               */
+  int max_ctas;  /* cap on the persistent grid (0 = one CTA per SM)                         */
+} cg_tuning_t;
+CG_API int cg_set_tuning(cg_handle_t h, const cg_tuning_t* t /* NULL = reset */);
+
+/* What the last successful cg_gemm_epilogue on this handle launched. */
+typedef struct cg_plan_info {
+  int tile_m, tile_n, cta_group, stages, group_m;
+  int grid;        /* CTAs launched                          */
+  int num_tiles;   /* output tiles                           */
+  int num_units;   /* k-block ranges (see cg_tuning)         */
+  int k_blocks;    /* 64-wide k-blocks per tile              */
+  int smem_bytes;  /* dynamic shared memory per CTA          */
+  int launches;    /* kernels launched by the call (always 1)*/
+} cg_plan_info_t;
+CG_API int cg_get_last_plan(cg_handle_t h, cg_plan_info_t* out);
+
+/*
+ * Copies a description of the last error into buf (NUL-terminated, at most len bytes).  With
+ * sync != 0 first synchronises the device and returns the device-side status word
+ * (CG_OK or CG_ERR_TIMEOUT), clearing it; with sync == 0 returns the last host-side status.
+ */
+CG_API int cg_last_error(cg_handle_t h, int sync, char* buf, size_t len);
+
+/* Frees the workspace and the handle.  The caller's tensors are not touched. */
+CG_API int cg_destroy(cg_handle_t h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CG_H_ */

@@ -1,0 +1,203 @@
+"""ctypes binding of libcg.so: the same names as the C ABI, argument marshalling only.
+
+Every step of the computation runs in the CUDA kernels of the library; there is no CPU or
+PyTorch fallback.  PyTorch appears only as the owner of device memory and streams: tensors
+are accepted wherever a device pointer is expected and their ``data_ptr()`` is passed on.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+from . import build as _build
+
+CG_OK, CG_ERR_INVALID_ARG, CG_ERR_UNSUPPORTED, CG_ERR_ARCH, CG_ERR_CUDA, CG_ERR_WORKSPACE, CG_ERR_TIMEOUT = range(7)
+CG_ACT_NONE, CG_ACT_RELU, CG_ACT_GELU_TANH, CG_ACT_SILU = 0, 1, 2, 3
+CG_FLAG_B_COLMAJOR = 1 << 8
+CG_FLAG_BIAS_BF16 = 1 << 9
+
+STATUS_NAMES = {0: "CG_OK", 1: "CG_ERR_INVALID_ARG", 2: "CG_ERR_UNSUPPORTED", 3: "CG_ERR_ARCH", 4: "CG_ERR_CUDA",
+                5: "CG_ERR_WORKSPACE", 6: "CG_ERR_TIMEOUT"}
+
+EXPORTS = ["cg_create", "cg_gemm_epilogue", "cg_gemm_epilogue_host", "cg_set_tuning", "cg_get_last_plan",
+           "cg_last_error", "cg_destroy"]
+
+
+class cg_tuning_t(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in ("tile_n", "cta_group", "num_units", "stages", "group_m", "max_ctas")]
+
+
+class cg_plan_info_t(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in ("tile_m", "tile_n", "cta_group", "stages", "group_m", "grid", "num_tiles",
+                                            "num_units", "k_blocks", "smem_bytes", "launches")]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_}
+
+
+class CgError(RuntimeError):
+    def __init__(self, code, msg=""):
+        super().__init__(f"{STATUS_NAMES.get(code, code)}: {msg}")
+        self.code = code
+
+
+_lib = None
+
+
+def lib_path() -> str:
+    return _build.LIB
+
+
+def load() -> ctypes.CDLL:
+    """Loads libcg.so, building it first when it is missing or older than its sources.
+    Raises if the library cannot be produced: there is nothing to fall back to."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.build()
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} is missing and could not be built; the CUDA library is required")
+    lib = ctypes.CDLL(path)
+    vp, ci, cf, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    lib.cg_create.argtypes = [ctypes.POINTER(vp), ci, sz]
+    gemm_args = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, cf, cf, ci, vp]
+    lib.cg_gemm_epilogue.argtypes = gemm_args
+    lib.cg_gemm_epilogue_host.argtypes = gemm_args
+    lib.cg_set_tuning.argtypes = [vp, ctypes.POINTER(cg_tuning_t)]
+    lib.cg_get_last_plan.argtypes = [vp, ctypes.POINTER(cg_plan_info_t)]
+    lib.cg_last_error.argtypes = [vp, ci, ctypes.c_char_p, sz]
+    lib.cg_destroy.argtypes = [vp]
+    for name in EXPORTS:
+        getattr(lib, name).restype = ci
+    _lib = lib
+    return lib
+
+
+def _dev_ptr(x) -> Optional[int]:
+    """torch CUDA tensor, int address or None -> address."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if hasattr(x, "data_ptr"):
+        if not x.is_cuda:
+            raise TypeError("expected a CUDA tensor (use cg_gemm_epilogue_host for host buffers)")
+        if not x.is_contiguous():
+            raise TypeError("tensors must be contiguous")
+        return x.data_ptr()
+    raise TypeError(f"cannot take a device pointer from {type(x)}")
+
+
+def _host_ptr(x) -> Optional[int]:
+    """numpy array, CPU torch tensor, int address or None -> address."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if hasattr(x, "data_ptr"):
+        if x.is_cuda or not x.is_contiguous():
+            raise TypeError("expected a contiguous CPU tensor")
+        return x.data_ptr()
+    if hasattr(x, "ctypes"):
+        if not x.flags.c_contiguous:
+            raise TypeError("arrays must be C-contiguous")
+        return x.ctypes.data
+    raise TypeError(f"cannot take a host pointer from {type(x)}")
+
+
+def _stream_ptr(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def cg_create(device: int = 0, workspace_bytes: int = 0) -> int:
+    h = ctypes.c_void_p()
+    rc = load().cg_create(ctypes.byref(h), int(device), int(workspace_bytes))
+    if rc != CG_OK:
+        raise CgError(rc, "cg_create failed")
+    return h.value
+
+
+def cg_gemm_epilogue(h, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, stream=None) -> int:
+    """Returns the status code (CG_OK = 0); raises nothing, like the C call."""
+    return load().cg_gemm_epilogue(h, _dev_ptr(A), _dev_ptr(B), _dev_ptr(bias), _dev_ptr(R), _dev_ptr(D), int(M), int(N),
+                                   int(K), int(batch), float(alpha), float(beta), int(act), _stream_ptr(stream))
+
+
+def cg_gemm_epilogue_host(h, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, stream=None) -> int:
+    return load().cg_gemm_epilogue_host(h, _host_ptr(A), _host_ptr(B), _host_ptr(bias), _host_ptr(R), _host_ptr(D),
+                                        int(M), int(N), int(K), int(batch), float(alpha), float(beta), int(act),
+                                        _stream_ptr(stream))
+
+
+def cg_set_tuning(h, tile_n=0, cta_group=0, num_units=0, stages=0, group_m=0, max_ctas=0, reset=False) -> int:
+    if reset:
+        return load().cg_set_tuning(h, None)
+    t = cg_tuning_t(tile_n, cta_group, num_units, stages, group_m, max_ctas)
+    return load().cg_set_tuning(h, ctypes.byref(t))
+
+
+def cg_get_last_plan(h) -> dict:
+    info = cg_plan_info_t()
+    rc = load().cg_get_last_plan(h, ctypes.byref(info))
+    if rc != CG_OK:
+        raise CgError(rc, "cg_get_last_plan failed")
+    return info.as_dict()
+
+
+def cg_last_error(h, sync: bool = False):
+    """Returns (status code, message)."""
+    buf = ctypes.create_string_buffer(256)
+    rc = load().cg_last_error(h, 1 if sync else 0, buf, 256)
+    return rc, buf.value.decode(errors="replace")
+
+
+def cg_destroy(h) -> int:
+    return load().cg_destroy(h)
+
+
+class Context:
+    """Small convenience wrapper: owns a handle, raises CgError on a non-zero status."""
+
+    def __init__(self, device: int = 0, workspace_bytes: int = 0):
+        self.handle = cg_create(device, workspace_bytes)
+
+    def gemm_epilogue(self, A, B, bias, R, D, M, N, K, batch=1, alpha=1.0, beta=0.0, act=CG_ACT_NONE, stream=None):
+        rc = cg_gemm_epilogue(self.handle, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, stream)
+        if rc != CG_OK:
+            raise CgError(rc, cg_last_error(self.handle)[1])
+
+    def gemm_epilogue_host(self, A, B, bias, R, D, M, N, K, batch=1, alpha=1.0, beta=0.0, act=CG_ACT_NONE, stream=None):
+        rc = cg_gemm_epilogue_host(self.handle, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, stream)
+        if rc != CG_OK:
+            raise CgError(rc, cg_last_error(self.handle)[1])
+
+    def set_tuning(self, **kw):
+        rc = cg_set_tuning(self.handle, **kw)
+        if rc != CG_OK:
+            raise CgError(rc, cg_last_error(self.handle)[1])
+
+    def last_plan(self) -> dict:
+        return cg_get_last_plan(self.handle)
+
+    def check(self):
+        """Synchronises and raises if the device reported an error (a bounded wait expired)."""
+        rc, msg = cg_last_error(self.handle, sync=True)
+        if rc != CG_OK:
+            raise CgError(rc, msg)
+
+    def close(self):
+        if self.handle:
+            cg_destroy(self.handle)
+            self.handle = None
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()

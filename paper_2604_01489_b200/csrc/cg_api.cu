@@ -1,0 +1,469 @@
+// C ABI of the cg library (see include/cg.h): argument validation, plan selection, tensor-map
+// encoding and the single kernel launch.  No CUDA library other than the runtime is called;
+// the driver's tensor-map encoder is fetched through the runtime's entry-point query.
+#include "../../include/cg.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdarg>
+#include <cstdint>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+
+#include "cg_kernel.cuh"
+
+namespace {
+
+using namespace cg;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+constexpr size_t DEFAULT_WORKSPACE = 64ull << 20;
+constexpr int MAX_TICKET_TILES = 1 << 16;          // tiles that may be split (4 tickets each)
+
+struct Plan {
+  int bn, cg, stages, group_m, num_units, grid, num_workers;
+  int tiles_m, tiles_n, num_tiles, k_blocks, smem;
+  bool b_kmajor;
+};
+
+struct StagingBuf {
+  void* ptr = nullptr;
+  size_t cap = 0;
+};
+
+}  // namespace
+
+struct cg_context {
+  int device = 0;
+  int num_sms = 0;
+  size_t workspace_bytes = 0;
+  uint8_t* workspace = nullptr;   // [tickets | partials]
+  int* tickets = nullptr;
+  float* partials = nullptr;
+  size_t partial_bytes = 0;
+  int* status = nullptr;
+  EncodeTiledFn encode = nullptr;
+  cg_tuning_t tuning{};
+  cg_plan_info_t last_plan{};
+  int last_status = CG_OK;
+  char last_msg[256] = {0};
+  long long wait_limit = 4000000000ll;   // about two seconds of SM clocks
+  int max_pairs = 0;                     // co-resident CTA pairs, filled lazily per kernel
+  StagingBuf sA, sB, sBias, sR, sD;
+  std::mutex mu;
+};
+
+namespace {
+
+int fail(cg_context* h, int code, const char* fmt, ...) {
+  if (h) {
+    h->last_status = code;
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(h->last_msg, sizeof h->last_msg, fmt, ap);
+    va_end(ap);
+  }
+  return code;
+}
+
+#define CG_CUDA(h, call)                                                                  \
+  do {                                                                                    \
+    cudaError_t e__ = (call);                                                             \
+    if (e__ != cudaSuccess) return fail(h, CG_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e__)); \
+  } while (0)
+
+int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// ---- kernel table ------------------------------------------------------------------
+
+typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const KernelParams);
+
+struct KernelEntry {
+  KernelFn fn;
+  int stage_bytes, fixed_bytes, stages_max;
+};
+
+template <int BN, int CGN, bool KM>
+KernelEntry entry() {
+  using C = Cfg<BN, CGN, KM>;
+  return KernelEntry{gemm_epilogue_kernel<BN, CGN, KM>, C::STAGE_BYTES, C::FIXED_BYTES, C::STAGES_MAX};
+}
+
+// index: [bn_idx (64,128,256)][cg-1][b_kmajor]
+bool lookup(int bn, int cgn, bool km, KernelEntry* out) {
+  if (cgn == 1) {
+    if (bn == 64) { *out = km ? entry<64, 1, true>() : entry<64, 1, false>(); return true; }
+    if (bn == 128) { *out = km ? entry<128, 1, true>() : entry<128, 1, false>(); return true; }
+    if (bn == 256) { *out = km ? entry<256, 1, true>() : entry<256, 1, false>(); return true; }
+  } else if (cgn == 2) {
+    if (bn == 128) { *out = km ? entry<128, 2, true>() : entry<128, 2, false>(); return true; }
+    if (bn == 256) { *out = km ? entry<256, 2, true>() : entry<256, 2, false>(); return true; }
+  }
+  return false;
+}
+
+int prepare_kernels(cg_context* h) {
+  const int bns[3] = {64, 128, 256};
+  for (int cgn = 1; cgn <= 2; ++cgn)
+    for (int i = 0; i < 3; ++i)
+      for (int km = 0; km < 2; ++km) {
+        KernelEntry e;
+        if (!lookup(bns[i], cgn, km != 0, &e)) continue;
+        CG_CUDA(h, cudaFuncSetAttribute(reinterpret_cast<const void*>(e.fn), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        SMEM_LIMIT));
+      }
+  return CG_OK;
+}
+
+// ---- tensor maps -------------------------------------------------------------------
+
+// bf16, rank 3 (inner, rows, batch), 128-byte swizzle, zero fill outside the tensor.
+int make_map(cg_context* h, CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows, uint64_t batch,
+             uint32_t box_inner, uint32_t box_rows) {
+  const cuuint64_t dims[3] = {inner, rows, batch};
+  const cuuint64_t strides[2] = {inner * 2, inner * rows * 2};
+  const cuuint32_t box[3] = {box_inner, box_rows, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = h->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box,
+                               estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS)
+    return fail(h, CG_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d) for dims %llu x %llu x %llu box %u x %u", (int)r,
+                (unsigned long long)inner, (unsigned long long)rows, (unsigned long long)batch, box_inner, box_rows);
+  return CG_OK;
+}
+
+// ---- plan --------------------------------------------------------------------------
+
+size_t partial_need(int num_units, int bn) { return static_cast<size_t>(2) * num_units * BM * bn * sizeof(float); }
+
+int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, Plan* pl) {
+  const cg_tuning_t& t = h->tuning;
+  const int sms = (t.max_ctas > 0 && t.max_ctas < h->num_sms) ? t.max_ctas : h->num_sms;
+  const int k_blocks = ceil_div(K, BK);
+  auto tiles = [&](int bm, int bn) -> long long {
+    return static_cast<long long>(batch) * ceil_div(M, bm) * ceil_div(N, bn);
+  };
+
+  int cgn = t.cta_group, bn = t.tile_n;
+  if (cgn == 0) {
+    // CTA pairs halve B's shared-memory traffic per flop; worth it once the machine is full
+    const int bn2 = bn ? bn : 256;
+    cgn = (M > BM && N >= 128 && bn2 >= 128 && tiles(2 * BM, bn2) >= sms) ? 2 : 1;
+  }
+  if (bn == 0) {
+    if (cgn == 2) {
+      bn = (N >= 256) ? 256 : 128;
+    } else {
+      // widest tile that still gives every SM a tile; otherwise the narrowest
+      bn = 64;
+      if (N >= 128 && tiles(BM, 128) >= sms) bn = 128;
+      if (N >= 256 && tiles(BM, 256) >= sms) bn = 256;
+    }
+  }
+  KernelEntry e;
+  if (!lookup(bn, cgn, b_kmajor, &e)) return fail(h, CG_ERR_INVALID_ARG, "no kernel for tile_n=%d cta_group=%d", bn, cgn);
+
+  pl->bn = bn;
+  pl->cg = cgn;
+  pl->b_kmajor = b_kmajor;
+  pl->k_blocks = k_blocks;
+  pl->tiles_m = ceil_div(M, BM * cgn);
+  pl->tiles_n = ceil_div(N, bn);
+  const long long nt = static_cast<long long>(batch) * pl->tiles_m * pl->tiles_n;
+  if (nt * k_blocks >= (1ll << 31) || nt >= (1ll << 29))
+    return fail(h, CG_ERR_UNSUPPORTED, "problem too large: %lld tiles x %d k-blocks", nt, k_blocks);
+  pl->num_tiles = static_cast<int>(nt);
+  const long long iters = nt * k_blocks;
+
+  int max_workers = sms / cgn;
+  if (max_workers < 1) max_workers = 1;
+
+  // units: data-parallel unless forced, or unless the tiles cannot fill the machine
+  long long units = pl->num_tiles;
+  if (t.num_units > 0) {
+    units = t.num_units;
+  } else if (cgn == 1 && pl->num_tiles < max_workers && k_blocks >= 8 && pl->num_tiles <= MAX_TICKET_TILES) {
+    // stream-K: one contiguous range per SM, at least 4 k-blocks each
+    long long u = max_workers;
+    if (u > iters / 4) u = iters / 4;
+    if (u > pl->num_tiles && partial_need(static_cast<int>(u), bn) <= h->partial_bytes) units = u;
+  }
+  if (units > iters) units = iters;
+  if (units < 1) units = 1;
+  if (units != pl->num_tiles) {
+    if (cgn != 1) return fail(h, CG_ERR_UNSUPPORTED, "split plans need cta_group 1");
+    if (pl->num_tiles > MAX_TICKET_TILES || partial_need(static_cast<int>(units), bn) > h->partial_bytes)
+      return fail(h, CG_ERR_WORKSPACE, "split plan needs %zu bytes of workspace, handle has %zu",
+                  partial_need(static_cast<int>(units), bn), h->partial_bytes);
+  }
+  pl->num_units = static_cast<int>(units);
+  pl->num_workers = pl->num_units < max_workers ? pl->num_units : max_workers;
+  pl->grid = pl->num_workers * cgn;
+
+  int stages = t.stages > 0 ? t.stages : e.stages_max;
+  if (stages > e.stages_max) stages = e.stages_max;
+  if (stages < 1) stages = 1;
+  pl->stages = stages;
+  pl->smem = stages * e.stage_bytes + e.fixed_bytes;
+
+  int gm = t.group_m > 0 ? t.group_m : 8;
+  if (gm > pl->tiles_m) gm = pl->tiles_m;
+  pl->group_m = gm;
+  return CG_OK;
+}
+
+int validate(cg_context* h, const void* A, const void* B, const void* bias, const void* R, void* D, int M, int N,
+             int K, int batch, float beta, int act) {
+  (void)bias;
+  if (!h) return CG_ERR_INVALID_ARG;
+  if (!A || !B || !D) return fail(h, CG_ERR_INVALID_ARG, "A, B and D must not be NULL");
+  if (M < 1 || N < 1 || K < 1 || batch < 1) return fail(h, CG_ERR_INVALID_ARG, "M, N, K, batch must be >= 1");
+  const int kind = act & 0xFF;
+  if (kind > CG_ACT_SILU || (act & ~(0xFF | CG_FLAG_B_COLMAJOR | CG_FLAG_BIAS_BF16)) != 0 || act < 0)
+    return fail(h, CG_ERR_INVALID_ARG, "unknown activation or flag bits in act=0x%x", act);
+  if (beta != 0.0f && !R) return fail(h, CG_ERR_INVALID_ARG, "R must not be NULL when beta != 0");
+  if (N % 8 != 0 || K % 8 != 0) return fail(h, CG_ERR_UNSUPPORTED, "N and K must be multiples of 8 (got N=%d K=%d)", N, K);
+  return CG_OK;
+}
+
+int check_alignment(cg_context* h, const void* A, const void* B, const void* bias, const void* R, void* D, float beta,
+                    int act) {
+  auto mis = [](const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0; };
+  if (mis(A, 16) || mis(B, 16) || mis(D, 16) || (beta != 0.0f && mis(R, 16)))
+    return fail(h, CG_ERR_UNSUPPORTED, "A, B, R and D must be 16-byte aligned");
+  if (bias && mis(bias, (act & CG_FLAG_BIAS_BF16) ? 2 : 4)) return fail(h, CG_ERR_UNSUPPORTED, "bias is misaligned");
+  return CG_OK;
+}
+
+int launch(cg_context* h, const void* A, const void* B, const void* bias, const void* R, void* D, int M, int N, int K,
+           int batch, float alpha, float beta, int act, cudaStream_t stream) {
+  const bool b_kmajor = (act & CG_FLAG_B_COLMAJOR) != 0;
+  Plan pl;
+  int rc = make_plan(h, M, N, K, batch, b_kmajor, &pl);
+  if (rc != CG_OK) return rc;
+  KernelEntry e;
+  lookup(pl.bn, pl.cg, b_kmajor, &e);
+
+  CUtensorMap tmA, tmB, tmD;
+  const int bn_cta = pl.bn / pl.cg;
+  if ((rc = make_map(h, &tmA, A, K, M, batch, BK, BM)) != CG_OK) return rc;
+  if (b_kmajor) rc = make_map(h, &tmB, B, K, N, batch, BK, bn_cta);
+  else rc = make_map(h, &tmB, B, N, K, batch, 64, BK);
+  if (rc != CG_OK) return rc;
+  if ((rc = make_map(h, &tmD, D, N, M, batch, EPI_COLS, 32)) != CG_OK) return rc;
+
+  KernelParams p;
+  memset(&p, 0, sizeof p);
+  p.M = M; p.N = N; p.K = K; p.batch = batch;
+  p.tiles_m = pl.tiles_m; p.tiles_n = pl.tiles_n; p.num_tiles = pl.num_tiles;
+  p.k_blocks = pl.k_blocks;
+  p.group_m = pl.group_m;
+  p.num_units = pl.num_units;
+  const long long iters = static_cast<long long>(pl.num_tiles) * pl.k_blocks;
+  p.unit_q = static_cast<int>(iters / pl.num_units);
+  p.unit_r = static_cast<int>(iters % pl.num_units);
+  p.num_workers = pl.num_workers;
+  p.stages = pl.stages;
+  p.alpha = alpha; p.beta = beta;
+  p.act = act & 0xFF;
+  p.bias_bf16 = (act & CG_FLAG_BIAS_BF16) ? 1 : 0;
+  p.bias = bias;
+  p.R = (beta != 0.0f) ? static_cast<const __nv_bfloat16*>(R) : nullptr;
+  p.partials = h->partials;
+  p.tickets = h->tickets;
+  p.status = h->status;
+  p.wait_limit = h->wait_limit;
+
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = dim3(pl.grid, 1, 1);
+  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = pl.smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = pl.cg;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  void* args[4] = {&tmA, &tmB, &tmD, &p};
+  CG_CUDA(h, cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(e.fn), args));
+
+  cg_plan_info_t& lp = h->last_plan;
+  lp.tile_m = BM * pl.cg; lp.tile_n = pl.bn; lp.cta_group = pl.cg; lp.stages = pl.stages; lp.group_m = pl.group_m;
+  lp.grid = pl.grid; lp.num_tiles = pl.num_tiles; lp.num_units = pl.num_units; lp.k_blocks = pl.k_blocks;
+  lp.smem_bytes = pl.smem; lp.launches = 1;
+  h->last_status = CG_OK;
+  h->last_msg[0] = 0;
+  if (getenv("CG_LOG"))
+    fprintf(stderr, "[cg] M=%d N=%d K=%d batch=%d tile=%dx%d cg=%d stages=%d group_m=%d grid=%d tiles=%d units=%d smem=%d\n", M,
+            N, K, batch, lp.tile_m, lp.tile_n, lp.cta_group, lp.stages, lp.group_m, lp.grid, lp.num_tiles, lp.num_units,
+            lp.smem_bytes);
+  return CG_OK;
+}
+
+int grow(cg_context* h, StagingBuf* s, size_t bytes) {
+  if (bytes <= s->cap) return CG_OK;
+  if (s->ptr) CG_CUDA(h, cudaFree(s->ptr));
+  s->ptr = nullptr;
+  s->cap = 0;
+  CG_CUDA(h, cudaMalloc(&s->ptr, bytes));
+  s->cap = bytes;
+  return CG_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int cg_create(cg_handle_t* out, int device, size_t workspace_bytes) {
+  if (!out) return CG_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (cudaSetDevice(device) != cudaSuccess) return CG_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return CG_ERR_CUDA;
+  if (prop.major != 10 || prop.minor != 0) return CG_ERR_ARCH;
+  cg_context* h = new (std::nothrow) cg_context;
+  if (!h) return CG_ERR_CUDA;
+  h->device = device;
+  h->num_sms = prop.multiProcessorCount;
+
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+      qres != cudaDriverEntryPointSuccess) {
+    delete h;
+    return CG_ERR_CUDA;
+  }
+  h->encode = reinterpret_cast<EncodeTiledFn>(fn);
+
+  if (workspace_bytes == 0) workspace_bytes = DEFAULT_WORKSPACE;
+  const size_t ticket_bytes = static_cast<size_t>(MAX_TICKET_TILES) * 4 * sizeof(int);
+  if (workspace_bytes < ticket_bytes + (1u << 20)) workspace_bytes = ticket_bytes + (1u << 20);
+  h->workspace_bytes = workspace_bytes;
+  if (cudaMalloc(reinterpret_cast<void**>(&h->workspace), workspace_bytes) != cudaSuccess ||
+      cudaMalloc(reinterpret_cast<void**>(&h->status), sizeof(int)) != cudaSuccess ||
+      cudaMemset(h->workspace, 0, ticket_bytes) != cudaSuccess || cudaMemset(h->status, 0, sizeof(int)) != cudaSuccess ||
+      prepare_kernels(h) != CG_OK) {
+    if (h->workspace) cudaFree(h->workspace);
+    if (h->status) cudaFree(h->status);
+    delete h;
+    return CG_ERR_CUDA;
+  }
+  h->tickets = reinterpret_cast<int*>(h->workspace);
+  h->partials = reinterpret_cast<float*>(h->workspace + ticket_bytes);
+  h->partial_bytes = workspace_bytes - ticket_bytes;
+  if (const char* w = getenv("CG_WAIT_LIMIT_CYCLES")) {
+    const long long v = atoll(w);
+    if (v > 0) h->wait_limit = v;
+  }
+  *out = h;
+  return CG_OK;
+}
+
+int cg_gemm_epilogue(cg_handle_t h, const void* A, const void* B, const void* bias, const void* R, void* D, int M,
+                     int N, int K, int batch, float alpha, float beta, int act, void* stream) {
+  if (!h) return CG_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(h->mu);
+  int rc = validate(h, A, B, bias, R, D, M, N, K, batch, beta, act);
+  if (rc != CG_OK) return rc;
+  if ((rc = check_alignment(h, A, B, bias, R, D, beta, act)) != CG_OK) return rc;
+  return launch(h, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, static_cast<cudaStream_t>(stream));
+}
+
+int cg_gemm_epilogue_host(cg_handle_t h, const void* A, const void* B, const void* bias, const void* R, void* D, int M,
+                          int N, int K, int batch, float alpha, float beta, int act, void* stream) {
+  if (!h) return CG_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(h->mu);
+  int rc = validate(h, A, B, bias, R, D, M, N, K, batch, beta, act);
+  if (rc != CG_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t a_bytes = static_cast<size_t>(batch) * M * K * 2, b_bytes = static_cast<size_t>(batch) * K * N * 2;
+  const size_t d_bytes = static_cast<size_t>(batch) * M * N * 2;
+  const size_t bias_bytes = bias ? static_cast<size_t>(N) * ((act & CG_FLAG_BIAS_BF16) ? 2 : 4) : 0;
+  const bool use_r = beta != 0.0f;
+  if ((rc = grow(h, &h->sA, a_bytes)) != CG_OK || (rc = grow(h, &h->sB, b_bytes)) != CG_OK ||
+      (rc = grow(h, &h->sD, d_bytes)) != CG_OK || (bias && (rc = grow(h, &h->sBias, bias_bytes)) != CG_OK) ||
+      (use_r && (rc = grow(h, &h->sR, d_bytes)) != CG_OK))
+    return rc;
+  CG_CUDA(h, cudaMemcpyAsync(h->sA.ptr, A, a_bytes, cudaMemcpyHostToDevice, st));
+  CG_CUDA(h, cudaMemcpyAsync(h->sB.ptr, B, b_bytes, cudaMemcpyHostToDevice, st));
+  if (bias) CG_CUDA(h, cudaMemcpyAsync(h->sBias.ptr, bias, bias_bytes, cudaMemcpyHostToDevice, st));
+  if (use_r) CG_CUDA(h, cudaMemcpyAsync(h->sR.ptr, R, d_bytes, cudaMemcpyHostToDevice, st));
+  rc = launch(h, h->sA.ptr, h->sB.ptr, bias ? h->sBias.ptr : nullptr, use_r ? h->sR.ptr : nullptr, h->sD.ptr, M, N, K,
+              batch, alpha, beta, act, st);
+  if (rc != CG_OK) return rc;
+  CG_CUDA(h, cudaMemcpyAsync(D, h->sD.ptr, d_bytes, cudaMemcpyDeviceToHost, st));
+  CG_CUDA(h, cudaStreamSynchronize(st));
+  return CG_OK;
+}
+
+int cg_set_tuning(cg_handle_t h, const cg_tuning_t* t) {
+  if (!h) return CG_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(h->mu);
+  if (!t) {
+    memset(&h->tuning, 0, sizeof h->tuning);
+    return CG_OK;
+  }
+  if ((t->tile_n != 0 && t->tile_n != 64 && t->tile_n != 128 && t->tile_n != 256) || t->cta_group < 0 ||
+      t->cta_group > 2 || t->num_units < 0 || t->stages < 0 || t->group_m < 0 || t->max_ctas < 0)
+    return fail(h, CG_ERR_INVALID_ARG, "bad tuning values");
+  h->tuning = *t;
+  return CG_OK;
+}
+
+int cg_get_last_plan(cg_handle_t h, cg_plan_info_t* out) {
+  if (!h || !out) return CG_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(h->mu);
+  *out = h->last_plan;
+  return CG_OK;
+}
+
+int cg_last_error(cg_handle_t h, int sync, char* buf, size_t len) {
+  if (!h) return CG_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(h->mu);
+  int code = h->last_status;
+  if (sync) {
+    int dev = 0;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpy(&dev, h->status, sizeof dev, cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess && dev != 0) e = cudaMemset(h->status, 0, sizeof(int));
+    if (e != cudaSuccess) {
+      code = fail(h, CG_ERR_CUDA, "device synchronisation failed: %s", cudaGetErrorString(e));
+    } else if (dev != 0) {
+      code = fail(h, dev, "a bounded wait inside the kernel expired (device status %d)", dev);
+      // a timed-out split tile may have left tickets behind
+      cudaMemset(h->tickets, 0, static_cast<size_t>(MAX_TICKET_TILES) * 4 * sizeof(int));
+    } else {
+      code = CG_OK;
+      if (h->last_status == CG_OK) h->last_msg[0] = 0;
+    }
+  }
+  if (buf && len > 0) {
+    strncpy(buf, h->last_msg, len - 1);
+    buf[len - 1] = 0;
+  }
+  return code;
+}
+
+int cg_destroy(cg_handle_t h) {
+  if (!h) return CG_ERR_INVALID_ARG;
+  cudaSetDevice(h->device);
+  cudaFree(h->workspace);
+  cudaFree(h->status);
+  StagingBuf* bufs[5] = {&h->sA, &h->sB, &h->sBias, &h->sR, &h->sD};
+  for (StagingBuf* s : bufs)
+    if (s->ptr) cudaFree(s->ptr);
+  delete h;
+  return CG_OK;
+}
+
+}  // extern "C"

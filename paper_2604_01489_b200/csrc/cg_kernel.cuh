@@ -1,0 +1,582 @@
+// Persistent, warp-specialised fused GEMM + epilogue kernel for sm_100a.
+//
+//   D[b,m,n] = act( alpha * sum_k A[b,m,k] * B[b,k,n] + bias[n] ) + beta * R[b,m,n]
+//
+// Roles inside one CTA of 192 threads:
+//   warp 0 (one lane)  producer: TMA loads of A and B k-blocks into an N-stage shared-memory
+//                      ring, completion counted in bytes on `full[stage]` mbarriers;
+//   warp 1 (one lane)  MMA issuer: tcgen05.mma (bf16 x bf16 -> fp32) from the ring into one of
+//                      two accumulator buffers in tensor memory; tcgen05.commit frees ring
+//                      stages (`empty[stage]`) and publishes accumulators (`acc_full[buf]`);
+//                      the whole warp allocates / frees tensor memory;
+//   warps 2-5          epilogue: TMEM -> registers, alpha*acc + bias, activation, + beta*R,
+//                      round to bf16, swizzled shared-memory staging, TMA store.  D is written
+//                      once and never read.  Each warp owns the 32 accumulator rows (TMEM
+//                      lanes) of its quarter and never synchronises with the other warps.
+//
+// Work decomposition: the iteration space (tile, k-block) is linearised tile-major and cut
+// into `num_units` contiguous, balanced ranges; worker w takes units w, w + W, ...  A unit
+// that covers whole tiles is plain data-parallel work; a unit boundary inside a tile makes
+// that tile split-K / stream-K: every contributor writes its fp32 partial to the workspace,
+// draws a ticket, and the last one to arrive sums all partials in unit order (deterministic)
+// and runs the epilogue.  Nobody ever waits for another CTA.
+//
+// With CG == 2 a pair of CTAs (cluster 2x1) shares one 256 x BN tile: each CTA loads its own
+// 128 rows of A and half of the B columns, the leader CTA issues tcgen05.mma.cta_group::2,
+// each CTA's epilogue drains its own 128 accumulator rows.
+//
+// Every wait is bounded: when a limit expires the CTA records CG_ERR_TIMEOUT in the status
+// word, raises a CTA-wide abort flag that all roles poll, and every role leaves its loop,
+// still frees tensor memory and returns.
+#pragma once
+
+#include <cuda_bf16.h>
+
+#include "cg_ptx.cuh"
+
+namespace cg {
+
+constexpr int BM = 128;          // accumulator rows per CTA (TMEM lanes)
+constexpr int BK = 64;           // k-block: 64 bf16 = one 128-byte swizzle row
+constexpr int UMMA_K = 16;       // K of one tcgen05.mma for 16-bit inputs
+constexpr int NUM_THREADS = 192;
+constexpr int MAX_STAGES = 12;
+constexpr int SMEM_LIMIT = 232448;  // 227 KiB opt-in maximum per CTA
+constexpr int EPI_COLS = 64;        // columns per epilogue chunk (one 128-byte bf16 row)
+constexpr int EPI_BUF_BYTES = 32 * EPI_COLS * 2;   // one warp's staging buffer: 32 rows x 128 B
+constexpr int EPI_BUFS = 2;
+constexpr int EPI_BYTES = 4 * EPI_BUFS * EPI_BUF_BYTES;
+constexpr int BIAS_BYTES = 4 * EPI_COLS * 4;       // per warp: one chunk of fp32 bias
+constexpr int CTRL_BYTES = 512;
+
+enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU_TANH = 2, ACT_SILU = 3 };
+enum { STATUS_OK = 0, STATUS_TIMEOUT = 6 };
+
+struct KernelParams {
+  int M, N, K, batch;
+  int tiles_m, tiles_n;   // tiles per batch entry; a tile is (CG*128) x BN
+  int num_tiles;
+  int k_blocks;           // ceil(K / 64)
+  int group_m;            // raster: m-tiles walked before the next n-tile
+  int num_units;          // contiguous k-block ranges
+  int unit_q, unit_r;     // start(u) = u*unit_q + min(u, unit_r)
+  int num_workers;        // CTAs (CG == 1) or CTA pairs (CG == 2)
+  int stages;
+  float alpha, beta;
+  int act;
+  int bias_bf16;
+  const void* bias;
+  const __nv_bfloat16* R;
+  float* partials;        // [2 * num_units][BM * BN] fp32 partial tiles
+  int* tickets;           // [num_tiles * 4], zero between launches
+  int* status;
+  long long wait_limit;   // clock cycles before a wait gives up
+};
+
+template <int BN, int CG, bool B_KMAJOR>
+struct Cfg {
+  static_assert(BN == 64 || BN == 128 || BN == 256, "tile width");
+  static_assert(CG == 1 || CG == 2, "cta group");
+  static constexpr int BN_CTA = BN / CG;                 // B columns each CTA loads
+  static constexpr int A_BYTES = BM * BK * 2;
+  static constexpr int B_BYTES = BN_CTA * BK * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int FIXED_BYTES = EPI_BYTES + BIAS_BYTES + CTRL_BYTES + 1024;  // + alignment slack
+  static constexpr int MAX_FIT = (SMEM_LIMIT - FIXED_BYTES) / STAGE_BYTES;
+  static constexpr int STAGES_MAX = MAX_FIT < MAX_STAGES ? MAX_FIT : MAX_STAGES;
+  static constexpr int TMEM_COLS = 2 * BN <= 32 ? 32 : (2 * BN <= 64 ? 64 : (2 * BN <= 128 ? 128 : (2 * BN <= 256 ? 256 : 512)));
+  static constexpr uint32_t IDESC = ptx::instr_desc_bf16(BM * CG, BN, !B_KMAJOR);
+  static constexpr int smem_bytes(int stages) { return stages * STAGE_BYTES + FIXED_BYTES; }
+};
+
+struct Ctrl {
+  uint64_t full[MAX_STAGES];
+  uint64_t empty[MAX_STAGES];
+  uint64_t acc_full[2];
+  uint64_t acc_empty[2];
+  uint64_t drain;
+  uint32_t tmem_base;
+  int abort;
+};
+static_assert(sizeof(Ctrl) <= CTRL_BYTES, "control block");
+
+// ---------------------------------------------------------------- scheduling helpers
+
+__device__ __forceinline__ int unit_start(const KernelParams& p, int u) {
+  return u * p.unit_q + (u < p.unit_r ? u : p.unit_r);
+}
+__device__ __forceinline__ int unit_of_iter(const KernelParams& p, int it) {
+  const int big = p.unit_r * (p.unit_q + 1);
+  return it < big ? it / (p.unit_q + 1) : p.unit_r + (it - big) / p.unit_q;
+}
+
+struct Segment {
+  int tile, kb0, kb1, unit;
+  bool head;   // first segment of its unit
+};
+
+// The sequence of (tile, k-range) segments a worker processes; all roles walk the same one.
+struct WorkIter {
+  const KernelParams& p;
+  int unit, it, end;
+  bool head;
+  __device__ WorkIter(const KernelParams& p_, int worker) : p(p_), unit(worker - p_.num_workers), it(0), end(0), head(false) {}
+  __device__ bool next(Segment& s) {
+    while (it >= end) {
+      unit += p.num_workers;
+      if (unit >= p.num_units) return false;
+      it = unit_start(p, unit);
+      end = unit_start(p, unit + 1);
+      head = true;
+    }
+    s.tile = it / p.k_blocks;
+    s.kb0 = it - s.tile * p.k_blocks;
+    int len = p.k_blocks - s.kb0;
+    if (len > end - it) len = end - it;
+    s.kb1 = s.kb0 + len;
+    s.unit = unit;
+    s.head = head;
+    head = false;
+    it += len;
+    return true;
+  }
+};
+
+// Linear tile id -> (batch, m-tile, n-tile): batch slowest, then groups of `group_m` m-tiles
+// walked down before stepping to the next n-tile, so that the tiles in flight at one time
+// share A rows and B columns in L2.
+__device__ __forceinline__ void decode_tile(const KernelParams& p, int tile, int& b, int& mt, int& nt) {
+  const int per_batch = p.tiles_m * p.tiles_n;
+  b = tile / per_batch;
+  const int r = tile - b * per_batch;
+  const int gsz = p.group_m * p.tiles_n;
+  const int g = r / gsz;
+  const int first_m = g * p.group_m;
+  int gm = p.tiles_m - first_m;
+  if (gm > p.group_m) gm = p.group_m;
+  const int rr = r - g * gsz;
+  nt = rr / gm;
+  mt = first_m + (rr - nt * gm);
+}
+
+// Bounded mbarrier wait.  false: gave up (limit expired here, or another role aborted).
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, Ctrl* ctrl, const KernelParams& p) {
+  if (ptx::mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (uint32_t spin = 1;; ++spin) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    if ((spin & 31u) == 0u) {
+      if (*reinterpret_cast<volatile int*>(&ctrl->abort)) return false;
+      if (clock64() - t0 > p.wait_limit) {
+        *reinterpret_cast<volatile int*>(&ctrl->abort) = 1;
+        atomicCAS(p.status, STATUS_OK, STATUS_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------- epilogue math
+
+template <int ACT>
+__device__ __forceinline__ float activate(float t) {
+  if constexpr (ACT == ACT_RELU) {
+    return fmaxf(t, 0.0f);
+  } else if constexpr (ACT == ACT_SILU) {
+    return __fdividef(t, 1.0f + __expf(-t));                         // t * sigmoid(t)
+  } else if constexpr (ACT == ACT_GELU_TANH) {
+    // 0.5 t (1 + tanh z) = t * sigmoid(2 z),  z = sqrt(2/pi) (t + 0.044715 t^3)
+    const float z2 = 1.5957691216057308f * (t + 0.044715f * t * t * t);
+    return __fdividef(t, 1.0f + __expf(-z2));
+  } else {
+    return t;
+  }
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);   // .x = lo (low half), .y = hi
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+
+// One warp, one 64-column chunk: acc (thread = row, 64 fp32) -> bf16 in swizzled staging.
+//   t = alpha*acc + bias[n];  u = act(t);  v = u + beta*R[m,n]
+template <int ACT, bool HAS_R>
+__device__ __forceinline__ void epilogue_chunk(const float (&acc)[EPI_COLS], const float* bias_s, float alpha,
+                                               float beta, const __nv_bfloat16* r_row, int n_valid,
+                                               bool row_valid, uint32_t stage_row_addr, int lane) {
+#pragma unroll
+  for (int c = 0; c < EPI_COLS / 8; ++c) {       // 8 columns = one 16-byte chunk of bf16
+    float v[8];
+    const float4 b0 = *reinterpret_cast<const float4*>(bias_s + c * 8);
+    const float4 b1 = *reinterpret_cast<const float4*>(bias_s + c * 8 + 4);
+    const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = activate<ACT>(fmaf(alpha, acc[c * 8 + j], bb[j]));
+    if constexpr (HAS_R) {
+      if (row_valid && c * 8 < n_valid) {
+        const uint4 rr = *reinterpret_cast<const uint4*>(r_row + c * 8);
+        const uint32_t w[4] = {rr.x, rr.y, rr.z, rr.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          v[2 * j] = fmaf(beta, __uint_as_float(w[j] << 16), v[2 * j]);
+          v[2 * j + 1] = fmaf(beta, __uint_as_float(w[j] & 0xFFFF0000u), v[2 * j + 1]);
+        }
+      }
+    }
+    const uint32_t o0 = pack_bf16x2(v[0], v[1]), o1 = pack_bf16x2(v[2], v[3]);
+    const uint32_t o2 = pack_bf16x2(v[4], v[5]), o3 = pack_bf16x2(v[6], v[7]);
+    // 128-byte swizzle: 16-byte chunk index XOR (row mod 8); staging rows are 128 B, row = lane
+    const uint32_t addr = stage_row_addr + (static_cast<uint32_t>(c ^ (lane & 7)) << 4);
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------- the kernel
+
+template <int BN, int CG, bool B_KMAJOR>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                     const __grid_constant__ CUtensorMap tmD, const KernelParams p) {
+  using C = Cfg<BN, CG, B_KMAJOR>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw_addr = ptx::smem_u32(smem_raw);
+  const uint32_t pad = ((raw_addr + 1023u) & ~1023u) - raw_addr;
+  uint8_t* smem = smem_raw + pad;                       // 1024-byte aligned (swizzle atoms)
+  const uint32_t ring_addr = raw_addr + pad;
+  const int stages = p.stages;
+  uint8_t* epi_ptr = smem + stages * C::STAGE_BYTES;
+  const uint32_t epi_addr = ring_addr + stages * C::STAGE_BYTES;
+  float* bias_all = reinterpret_cast<float*>(epi_ptr + EPI_BYTES);
+  Ctrl* ctrl = reinterpret_cast<Ctrl*>(epi_ptr + EPI_BYTES + BIAS_BYTES);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t cta_rank = (CG == 2) ? ptx::cluster_ctarank() : 0u;
+  const int worker = blockIdx.x / CG;
+
+  // ---- set-up: barriers, tensor memory
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      ptx::mbar_init(ptx::smem_u32(&ctrl->full[s]), 1);
+      ptx::mbar_init(ptx::smem_u32(&ctrl->empty[s]), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(ptx::smem_u32(&ctrl->acc_full[a]), 1);
+      ptx::mbar_init(ptx::smem_u32(&ctrl->acc_empty[a]), 4 * CG);   // one arrive per epilogue warp of the pair
+    }
+    ptx::mbar_init(ptx::smem_u32(&ctrl->drain), 1);
+    ctrl->abort = 0;
+    ptx::fence_mbar_init();
+    ptx::prefetch_tensormap(&tmA);
+    ptx::prefetch_tensormap(&tmB);
+    ptx::prefetch_tensormap(&tmD);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc<CG>(ptx::smem_u32(&ctrl->tmem_base), C::TMEM_COLS);
+    ptx::tmem_relinquish<CG>();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if constexpr (CG == 2) {   // the peer's barriers must exist before anything signals them
+    ptx::cluster_arrive();
+    ptx::cluster_wait();
+  }
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&ctrl->tmem_base);
+
+  if (warp == 0) {
+    // ================================================================ producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      WorkIter wi(p, worker);
+      Segment s;
+      bool ok = true;
+      uint32_t filled_mask = 0, filled_parity = 0;   // stages with a load in flight and the phase it completes
+      while (ok && wi.next(s)) {
+        int b, mt, nt;
+        decode_tile(p, s.tile, b, mt, nt);
+        const int m0 = mt * (BM * CG) + static_cast<int>(cta_rank) * BM;
+        const int n0 = nt * BN + static_cast<int>(cta_rank) * C::BN_CTA * (CG - 1);
+        for (int kb = s.kb0; kb < s.kb1; ++kb) {
+          if (!wait_bar(ptx::smem_u32(&ctrl->empty[stage]), phase ^ 1u, ctrl, p)) { ok = false; break; }
+          const uint32_t full_local = ptx::smem_u32(&ctrl->full[stage]);
+          const uint32_t a_dst = ring_addr + stage * C::STAGE_BYTES;
+          const uint32_t b_dst = a_dst + C::A_BYTES;
+          if constexpr (CG == 1) {
+            ptx::mbar_arrive_expect_tx(full_local, C::STAGE_BYTES);
+            ptx::tma_load_3d(a_dst, &tmA, full_local, kb * BK, m0, b);
+            if constexpr (B_KMAJOR) {
+              ptx::tma_load_3d(b_dst, &tmB, full_local, kb * BK, n0, b);
+            } else {
+#pragma unroll
+              for (int j = 0; j < C::BN_CTA / 64; ++j)
+                ptx::tma_load_3d(b_dst + j * (64 * BK * 2), &tmB, full_local, n0 + j * 64, kb * BK, b);
+            }
+          } else {
+            // both CTAs' bytes are counted on the leader's barrier
+            if (cta_rank == 0) ptx::mbar_arrive_expect_tx(full_local, 2 * C::STAGE_BYTES);
+            const uint32_t full_leader = ptx::mapa(full_local, 0);
+            ptx::tma_load_3d_pair(a_dst, &tmA, full_leader, kb * BK, m0, b);
+            if constexpr (B_KMAJOR) {
+              ptx::tma_load_3d_pair(b_dst, &tmB, full_leader, kb * BK, n0, b);
+            } else {
+#pragma unroll
+              for (int j = 0; j < C::BN_CTA / 64; ++j)
+                ptx::tma_load_3d_pair(b_dst + j * (64 * BK * 2), &tmB, full_leader, n0 + j * 64, kb * BK, b);
+            }
+          }
+          filled_mask |= 1u << stage;
+          filled_parity = (filled_parity & ~(1u << stage)) | (phase << stage);
+          if (++stage == stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok || *reinterpret_cast<volatile int*>(&ctrl->abort)) {
+        // abort path: let this CTA's own copies land before shared memory is given up
+        if (CG == 1 || cta_rank == 0) {
+          for (int s2 = 0; s2 < stages; ++s2)
+            if (filled_mask & (1u << s2)) {
+              const long long t0 = clock64();
+              while (!ptx::mbar_try_wait(ptx::smem_u32(&ctrl->full[s2]), (filled_parity >> s2) & 1u))
+                if (clock64() - t0 > p.wait_limit) break;
+            }
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ================================================================ MMA issuer
+    if (lane == 0 && (CG == 1 || cta_rank == 0)) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      WorkIter wi(p, worker);
+      Segment s;
+      bool ok = true;
+      while (ok && wi.next(s)) {
+        if (!wait_bar(ptx::smem_u32(&ctrl->acc_empty[acc]), acc_phase ^ 1u, ctrl, p)) { ok = false; break; }
+        ptx::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
+        for (int kb = s.kb0; kb < s.kb1; ++kb) {
+          if (!wait_bar(ptx::smem_u32(&ctrl->full[stage]), phase, ctrl, p)) { ok = false; break; }
+          ptx::tc_fence_after();
+          const uint32_t a_addr = ring_addr + stage * C::STAGE_BYTES;
+          const uint32_t b_addr = a_addr + C::A_BYTES;
+          int nk = (p.K - kb * BK + UMMA_K - 1) / UMMA_K;     // skip 16-wide steps that are all padding
+          if (nk > BK / UMMA_K) nk = BK / UMMA_K;
+          for (int k = 0; k < nk; ++k) {
+            // A, K-major: +16 elements along K = +32 bytes inside the 128-byte swizzle row
+            const uint64_t a_desc = ptx::smem_desc_sw128(a_addr + k * (UMMA_K * 2), 16, 8 * 128);
+            uint64_t b_desc;
+            if constexpr (B_KMAJOR) {
+              b_desc = ptx::smem_desc_sw128(b_addr + k * (UMMA_K * 2), 16, 8 * 128);
+            } else {
+              // B, N-major: rows are k, 128 B = 64 n; +16 k = two 8-row groups = +2048 bytes;
+              // 64-column blocks are whole TMA boxes, 64*64*2 bytes apart
+              b_desc = ptx::smem_desc_sw128(b_addr + k * (UMMA_K * 128), 64 * BK * 2, 8 * 128);
+            }
+            ptx::mma_f16<CG>(d_tmem, a_desc, b_desc, C::IDESC, (kb > s.kb0 || k > 0) ? 1u : 0u);
+          }
+          const uint32_t empty_local = ptx::smem_u32(&ctrl->empty[stage]);
+          ptx::tc_commit<CG>(empty_local);
+          if constexpr (CG == 2) ptx::tc_commit<CG>(ptx::mapa(empty_local, 1));
+          if (++stage == stages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        const uint32_t full_local = ptx::smem_u32(&ctrl->acc_full[acc]);
+        ptx::tc_commit<CG>(full_local);
+        if constexpr (CG == 2) ptx::tc_commit<CG>(ptx::mapa(full_local, 1));
+        acc ^= 1;
+        if (acc == 0) acc_phase ^= 1u;
+      }
+      if (!ok || *reinterpret_cast<volatile int*>(&ctrl->abort)) {
+        // abort path: wait (bounded) until the MMAs issued so far have retired
+        ptx::tc_commit<CG>(ptx::smem_u32(&ctrl->drain));
+        const long long t0 = clock64();
+        while (!ptx::mbar_try_wait(ptx::smem_u32(&ctrl->drain), 0))
+          if (clock64() - t0 > p.wait_limit) break;
+      }
+    }
+    __syncwarp();
+  } else {
+    // ================================================================ epilogue (warps 2..5)
+    const int q = warp & 3;                     // TMEM lane quarter this warp may access
+    const int row_in_tile = q * 32 + lane;
+    float* bias_s = bias_all + q * EPI_COLS;
+    const uint32_t stage_base = epi_addr + q * (EPI_BUFS * EPI_BUF_BYTES);
+    int store_buf = 0;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    WorkIter wi(p, worker);
+    Segment s;
+    bool ok = true;
+    const bool has_r = (p.beta != 0.0f);
+    while (ok && wi.next(s)) {
+      int b, mt, nt;
+      decode_tile(p, s.tile, b, mt, nt);
+      const int m_base = mt * (BM * CG) + static_cast<int>(cta_rank) * BM;   // first row of this CTA's slab
+      const int n_base = nt * BN;
+      const int m = m_base + row_in_tile;
+      const bool row_valid = m < p.M;
+      const bool warp_rows_valid = (m_base + q * 32) < p.M;
+      const bool whole_tile = (s.kb0 == 0 && s.kb1 == p.k_blocks);
+      if (!wait_bar(ptx::smem_u32(&ctrl->acc_full[acc]), acc_phase, ctrl, p)) { ok = false; break; }
+      ptx::tc_fence_after();
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(acc * BN);
+      const uint32_t acc_empty_bar = (CG == 2) ? ptx::mapa(ptx::smem_u32(&ctrl->acc_empty[acc]), 0)
+                                               : ptx::smem_u32(&ctrl->acc_empty[acc]);
+      int n_chunks = (p.N - n_base + EPI_COLS - 1) / EPI_COLS;    // chunks with at least one valid column
+      if (n_chunks > BN / EPI_COLS) n_chunks = BN / EPI_COLS;
+
+      bool reduce = false;        // this warp must run the epilogue from workspace partials
+      int first_unit = 0, last_unit = 0;
+      if (!whole_tile) {
+        // ---- split tile: park the fp32 partial, draw a ticket
+        const int slot = 2 * s.unit + (s.head ? 0 : 1);
+        float4* part = reinterpret_cast<float4*>(p.partials) + (static_cast<size_t>(slot) * (BM * BN / 4)) +
+                       static_cast<size_t>(q) * (32 * BN / 4);
+        for (int c = 0; c < BN / 32; ++c) {
+          uint32_t v[32];
+          ptx::tmem_ld_32x32b_x32(taddr + c * 32, v);
+          ptx::tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 8; ++j)   // float4 index j of this 32-column group; lanes contiguous
+            __stcg(part + (c * 8 + j) * 32 + lane,
+                   make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]),
+                               __uint_as_float(v[4 * j + 3])));
+        }
+        ptx::tc_fence_before();
+        __threadfence();
+        __syncwarp();
+        int last = 0;
+        if (lane == 0) {
+          if constexpr (CG == 2) ptx::mbar_arrive_cluster(acc_empty_bar); else ptx::mbar_arrive(acc_empty_bar);
+          first_unit = unit_of_iter(p, s.tile * p.k_blocks);
+          last_unit = unit_of_iter(p, (s.tile + 1) * p.k_blocks - 1);
+          const int parts = last_unit - first_unit + 1;
+          const int old = atomicAdd(p.tickets + s.tile * 4 + q, 1);
+          last = (old == parts - 1) ? 1 : 0;
+          if (last) {
+            __threadfence();
+            atomicExch(p.tickets + s.tile * 4 + q, 0);     // self-reset for the next launch
+          }
+        }
+        last = __shfl_sync(0xFFFFFFFFu, last, 0);
+        first_unit = __shfl_sync(0xFFFFFFFFu, first_unit, 0);
+        last_unit = __shfl_sync(0xFFFFFFFFu, last_unit, 0);
+        reduce = (last != 0);
+        if (reduce) __threadfence();
+      }
+
+      if (whole_tile || reduce) {
+        for (int c = 0; c < n_chunks; ++c) {
+          const int n0 = n_base + c * EPI_COLS;
+          int n_valid = p.N - n0;
+          if (n_valid > EPI_COLS) n_valid = EPI_COLS;
+          // bias for this chunk: two values per lane, staged per warp
+          float bv0 = 0.0f, bv1 = 0.0f;
+          if (p.bias != nullptr) {
+            if (p.bias_bf16) {
+              const __nv_bfloat16* bp = static_cast<const __nv_bfloat16*>(p.bias);
+              if (lane < n_valid) bv0 = __bfloat162float(bp[n0 + lane]);
+              if (lane + 32 < n_valid) bv1 = __bfloat162float(bp[n0 + lane + 32]);
+            } else {
+              const float* bp = static_cast<const float*>(p.bias);
+              if (lane < n_valid) bv0 = __ldg(bp + n0 + lane);
+              if (lane + 32 < n_valid) bv1 = __ldg(bp + n0 + lane + 32);
+            }
+          }
+          float accv[EPI_COLS];
+          if (whole_tile) {
+            uint32_t v0[32], v1[32];
+            ptx::tmem_ld_32x32b_x32(taddr + c * EPI_COLS, v0);
+            ptx::tmem_ld_32x32b_x32(taddr + c * EPI_COLS + 32, v1);
+            ptx::tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) { accv[j] = __uint_as_float(v0[j]); accv[32 + j] = __uint_as_float(v1[j]); }
+            if (c == n_chunks - 1) {     // accumulator fully read: hand the buffer back to the MMA warp
+              ptx::tc_fence_before();
+              __syncwarp();
+              if (lane == 0) {
+                if constexpr (CG == 2) ptx::mbar_arrive_cluster(acc_empty_bar); else ptx::mbar_arrive(acc_empty_bar);
+              }
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < EPI_COLS; ++j) accv[j] = 0.0f;
+            for (int u = first_unit; u <= last_unit; ++u) {     // fixed order => deterministic sum
+              const int slot = 2 * u + (unit_start(p, u) >= s.tile * p.k_blocks ? 0 : 1);
+              const float4* part = reinterpret_cast<const float4*>(p.partials) +
+                                   (static_cast<size_t>(slot) * (BM * BN / 4)) + static_cast<size_t>(q) * (32 * BN / 4);
+#pragma unroll
+              for (int j = 0; j < EPI_COLS / 4; ++j) {
+                const float4 t = __ldcg(part + (c * (EPI_COLS / 4) + j) * 32 + lane);
+                accv[4 * j] += t.x; accv[4 * j + 1] += t.y; accv[4 * j + 2] += t.z; accv[4 * j + 3] += t.w;
+              }
+            }
+          }
+          // staging buffer free again?  (the store issued two chunks ago has read it)
+          if (lane == 0) ptx::bulk_wait_group_read<EPI_BUFS - 1>();
+          __syncwarp();
+          bias_s[lane] = bv0;
+          bias_s[lane + 32] = bv1;
+          __syncwarp();
+          const uint32_t buf_addr = stage_base + store_buf * EPI_BUF_BYTES;
+          const uint32_t row_addr = buf_addr + lane * 128;
+          const __nv_bfloat16* r_row = has_r ? p.R + (static_cast<size_t>(b) * p.M + (row_valid ? m : 0)) * p.N + n0 : nullptr;
+          switch (p.act) {
+            case ACT_RELU:
+              if (has_r) epilogue_chunk<ACT_RELU, true>(accv, bias_s, p.alpha, p.beta, r_row, n_valid, row_valid, row_addr, lane);
+              else epilogue_chunk<ACT_RELU, false>(accv, bias_s, p.alpha, p.beta, r_row, n_valid, row_valid, row_addr, lane);
+              break;
+            case ACT_GELU_TANH:
+              if (has_r) epilogue_chunk<ACT_GELU_TANH, true>(accv, bias_s, p.alpha, p.beta, r_row, n_valid, row_valid, row_addr, lane);
+              else epilogue_chunk<ACT_GELU_TANH, false>(accv, bias_s, p.alpha, p.beta, r_row, n_valid, row_valid, row_addr, lane);
+              break;
+            case ACT_SILU:
+              if (has_r) epilogue_chunk<ACT_SILU, true>(accv, bias_s, p.alpha, p.beta, r_row, n_valid, row_valid, row_addr, lane);
+              else epilogue_chunk<ACT_SILU, false>(accv, bias_s, p.alpha, p.beta, r_row, n_valid, row_valid, row_addr, lane);
+              break;
+            default:
+              if (has_r) epilogue_chunk<ACT_NONE, true>(accv, bias_s, p.alpha, p.beta, r_row, n_valid, row_valid, row_addr, lane);
+              else epilogue_chunk<ACT_NONE, false>(accv, bias_s, p.alpha, p.beta, r_row, n_valid, row_valid, row_addr, lane);
+              break;
+          }
+          ptx::fence_proxy_async_smem();      // my generic-proxy writes -> visible to the TMA store
+          __syncwarp();
+          if (lane == 0) {
+            if (warp_rows_valid) ptx::tma_store_3d(&tmD, buf_addr, n0, m_base + q * 32, b);   // clips rows >= M, cols >= N
+            ptx::bulk_commit_group();
+          }
+          store_buf = (store_buf + 1 == EPI_BUFS) ? 0 : store_buf + 1;
+        }
+        if (whole_tile && n_chunks == 0) {   // cannot happen (n_base < N), kept for symmetry of the protocol
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) {
+            if constexpr (CG == 2) ptx::mbar_arrive_cluster(acc_empty_bar); else ptx::mbar_arrive(acc_empty_bar);
+          }
+        }
+      }
+      acc ^= 1;
+      if (acc == 0) acc_phase ^= 1u;
+    }
+    if (lane == 0) ptx::bulk_wait_group<0>();   // all of this warp's stores have completed
+    __syncwarp();
+  }
+
+  // ---- tear-down
+  ptx::tc_fence_before();
+  __syncthreads();
+  if constexpr (CG == 2) {   // neither CTA may retire while the other can still signal its barriers or use its TMEM
+    ptx::cluster_arrive();
+    ptx::cluster_wait();
+  }
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc<CG>(tmem_base, C::TMEM_COLS);
+  }
+}
+
+}  // namespace cg

@@ -1,0 +1,60 @@
+"""Helpers shared by the GPU parity tests: run one problem through the C ABI and compare the
+result with the CPU oracle on the same seeded inputs."""
+from __future__ import annotations
+
+import numpy as np
+
+from cg_inputs import gen, workloads as W
+
+ELEM_TOL = 1e-2      # |D_gpu - D_ref| <= ELEM_TOL * (|D_ref| + 1)   for every element
+FRO_TOL = 5e-3       # ||D_gpu - D_ref||_F / ||D_ref||_F
+
+
+def to_device(p, device="cuda:0"):
+    """Problem (numpy) -> dict of torch CUDA tensors; bf16 operands are bit-cast, not converted."""
+    import torch
+
+    def bf16(x):
+        return None if x is None else torch.from_numpy(x.view(np.int16)).to(device).view(torch.bfloat16)
+
+    bias = None
+    if p.bias is not None:
+        bias = bf16(p.bias) if p.act & W.FLAG_BIAS_BF16 else torch.from_numpy(p.bias).to(device)
+    d = torch.empty((p.batch, p.M, p.N), dtype=torch.bfloat16, device=device)
+    return dict(A=bf16(p.A), B=bf16(p.B), bias=bias, R=bf16(p.R), D=d)
+
+
+def run_gpu(ctx, p, dev=None, fill=None):
+    """One cg_gemm_epilogue call; returns D as uint16 bf16 bits [batch, M, N] (numpy)."""
+    import torch
+    if dev is None:
+        dev = to_device(p)
+    if fill is not None:
+        dev["D"].view(torch.int16).fill_(fill)
+    ctx.gemm_epilogue(dev["A"], dev["B"], dev["bias"], dev["R"], dev["D"], p.M, p.N, p.K, p.batch, p.alpha, p.beta, p.act)
+    ctx.check()
+    return dev["D"].view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def compare(d_bits, ref64, ref16=None):
+    """Error figures of bf16 bits `d_bits` against the fp64 oracle result `ref64` (same shape)."""
+    got = gen.bf16_bits_to_f32(d_bits).astype(np.float64).reshape(ref64.shape)
+    err = np.abs(got - ref64)
+    bound = ELEM_TOL * (np.abs(ref64) + 1.0)
+    worst = float(np.max(err / bound)) if err.size else 0.0
+    nref = float(np.linalg.norm(ref64))
+    fro = float(np.linalg.norm(got - ref64) / nref) if nref > 0 else float(np.max(np.abs(got)))
+    out = dict(worst_ratio=worst, rel_fro=fro, n_bad=int(np.sum(err > bound)), finite=bool(np.all(np.isfinite(got))))
+    if ref16 is not None:
+        out["bit_equal"] = bool(np.array_equal(d_bits.reshape(ref16.shape), ref16))
+        out["n_bits_differ"] = int(np.sum(d_bits.reshape(ref16.shape) != ref16))
+    out["ok"] = out["finite"] and out["n_bad"] == 0 and fro <= FRO_TOL
+    return out
+
+
+def oracle_full(oracle, p):
+    return oracle.gemm_epilogue(p.A, p.B, p.bias, p.R, p.M, p.N, p.K, p.batch, p.alpha, p.beta, p.act)
+
+
+def oracle_rows(oracle, p, rows):
+    return oracle.gemm_epilogue_rows(p.A, p.B, p.bias, p.R, rows, p.M, p.N, p.K, p.batch, p.alpha, p.beta, p.act)
