@@ -1,0 +1,351 @@
+#!/usr/bin/env python
+"""Benchmark of the fused bf16 GEMM + epilogue (C ABI: cg_gemm_epilogue) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
+
+One "step" is one call of the whole hot path (one kernel launch) on one seeded synthetic workload.
+Rank 0 prints ONE JSON line.  `value` is TFLOP/s (2*M*N*K*batch per step) with inputs resident in
+HBM; `e2e` is the same metric through cg_gemm_epilogue_host with pinned HOST buffers, copies inside
+the timed region.  With N > 1 (torchrun, one rank per GPU) every rank runs its own replica of the
+workload -- the path shards without any exchange, so there is no collective on the data path --
+and `value` sums the ranks' work over the slowest rank's time ("weak" scaling).
+
+`--impl reference` times the CPU oracle (as it stands, one core) on bounded row samples of the same
+workload: a deliberately slow baseline, not a target.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from cg_inputs import workloads as W  # noqa: E402
+
+METRIC = "fused bf16 GEMM+epilogue TFLOP/s"
+UNIT = "TFLOP/s"
+DEFAULT_CONFIG = "cfg5_8192_silu"      # the headline compute-bound shape of the metric
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
+# summarised under profiles/ (one capture per workload, heuristic plan).
+NCU_DRAM_TRAFFIC = {
+}
+
+BOUND = {"cfg1_256_relu": "latency", "cfg2_4096_gelu": "tensor", "cfg3_skinny_silu": "hbm",
+         "cfg4_batched_residual": "tensor", "cfg5_8192_silu": "tensor"}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d} | {"source": "measured"}
+    return dict(FALLBACK_PEAKS, source="fallback")
+
+
+def describe(p) -> str:
+    act = {0: "none", 1: "relu", 2: "gelu_tanh", 3: "silu"}[p.act & 0xFF]
+    lay = "B col-major" if p.act & W.FLAG_B_COLMAJOR else "B row-major"
+    bias = "no bias" if p.bias is None else ("bias bf16" if p.act & W.FLAG_BIAS_BF16 else "bias fp32")
+    return (f"{p.name}: M={p.M} N={p.N} K={p.K} batch={p.batch}, {lay}, {bias}, act={act}, alpha={p.alpha}, "
+            f"beta={p.beta}, seed={p.seed}")
+
+
+# ------------------------------------------------------------------ clocks
+
+class ClockSampler:
+    """Polls SM clock and throttle reasons through NVML (read-only) while a region runs."""
+
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, index: int, period_s: float = 0.002):
+        self.samples, self.reason_bits = [], 0
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.dev = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.dev, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+        self.period = period_s
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                self.samples.append(float(self.nv.nvmlDeviceGetClockInfo(self.dev, self.nv.NVML_CLOCK_SM)))
+                self.reason_bits |= int(self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.dev))
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=1.0)
+
+    def summary(self) -> dict:
+        reasons = [name for bit, name in self.REASONS.items() if self.reason_bits & bit]
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": reasons, "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------ reference arm (CPU oracle)
+
+def oracle_sample(p, nrows: int):
+    """Times the oracle, unchanged and single-threaded, on `nrows` seeded rows of the workload."""
+    from oracle import ref
+    ref.build()
+    rows = W.sample_rows(p, nrows)
+    t0 = time.perf_counter()
+    ref.gemm_epilogue_rows(p.A, p.B, p.bias, p.R, rows, p.M, p.N, p.K, p.batch, p.alpha, p.beta, p.act)
+    dt = time.perf_counter() - t0
+    flops = 2.0 * len(rows) * p.N * p.K
+    return dt, flops, len(rows)
+
+
+def rows_for_seconds(p, seconds: float) -> int:
+    """Row count whose oracle time is about `seconds` (calibrated on a few rows)."""
+    dt, _, n = oracle_sample(p, 4)
+    per_row = max(dt / n, 1e-6)
+    return int(max(1, min(p.batch * p.M, seconds / per_row)))
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    p = W.config(args.config)
+    nrows = rows_for_seconds(p, 0.5)
+    for _ in range(args.warmup):
+        oracle_sample(p, nrows)
+    total_t, total_f = 0.0, 0.0
+    for _ in range(args.steps):
+        dt, fl, _ = oracle_sample(p, nrows)
+        total_t += dt
+        total_f += fl
+    value = total_f / total_t / 1e12
+    sample = f"{nrows} of {p.batch * p.M} output rows per step (all N columns, full K), single-threaded fp64"
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": total_t / args.steps * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "impl": "reference",
+            "config": {"workload": describe(p), "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------ our arm
+
+def to_device(p, device):
+    import torch
+
+    def bf16(x):
+        return None if x is None else torch.from_numpy(x.view(np.int16)).to(device).view(torch.bfloat16)
+
+    bias = None
+    if p.bias is not None:
+        bias = bf16(p.bias) if p.act & W.FLAG_BIAS_BF16 else torch.from_numpy(p.bias).to(device)
+    return dict(A=bf16(p.A), B=bf16(p.B), bias=bias, R=bf16(p.R),
+                D=torch.empty((p.batch, p.M, p.N), dtype=torch.bfloat16, device=device))
+
+
+def pinned(x):
+    import torch
+    return None if x is None else torch.from_numpy(x.view(np.int16) if x.dtype == np.uint16 else x).pin_memory()
+
+
+def per_launch_times(ctx, p, dev, iters, flush):
+    """Each launch timed alone with CUDA events on the launching stream; L2 flushed in between."""
+    import torch
+    ts = []
+    for _ in range(iters):
+        if flush is not None:
+            flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ctx.gemm_epilogue(dev["A"], dev["B"], dev["bias"], dev["R"], dev["D"], p.M, p.N, p.K, p.batch, p.alpha, p.beta, p.act)
+        e1.record()
+        e1.synchronize()
+        ts.append(e0.elapsed_time(e1) * 1e-3)
+    return ts
+
+
+def workload_table(ctx, device, peaks, names):
+    """All five workloads, each launch timed alone after an L2 flush (their inputs may fit in L2)."""
+    import torch
+    flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=device)
+    out = {}
+    for name in names:
+        p = W.config(name)
+        dev = to_device(p, device)
+        per_launch_times(ctx, p, dev, 3, flush)
+        ts = per_launch_times(ctx, p, dev, 20, flush)
+        ctx.check()
+        best, med = min(ts), float(np.median(ts))
+        row = {"us_best": best * 1e6, "us_median": med * 1e6, "tflops_best": p.flops / best / 1e12,
+               "tflops_median": p.flops / med / 1e12, "gbs_best": p.algorithmic_bytes / best / 1e9,
+               "frac_tensor_of_measured_burst": p.flops / best / 1e12 / peaks["bf16_tflops"],
+               "frac_tensor_of_nominal_2250": p.flops / best / 1e12 / 2250.0,
+               "frac_hbm_of_measured": p.algorithmic_bytes / best / 1e9 / peaks["hbm_gbs"],
+               "bound": BOUND[name], "plan": ctx.last_plan()}
+        out[name] = row
+        del dev
+    return out
+
+
+def run_ours(args):
+    import torch
+    import paper_2604_01489_b200 as cg
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    peaks = load_peaks()
+    p = W.config(args.config)                      # seeded host buffers (the same ones the oracle would read)
+    dev = to_device(p, device)
+    ctx = cg.Context(local_rank)
+    launch = lambda: ctx.gemm_epilogue(dev["A"], dev["B"], dev["bias"], dev["R"], dev["D"], p.M, p.N, p.K, p.batch,
+                                       p.alpha, p.beta, p.act)
+    footprint = p.algorithmic_bytes
+    flush = None
+    if footprint <= 2 * L2_BYTES:                  # inputs could sit in L2: flush between timed launches
+        flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=device)
+
+    for _ in range(max(args.warmup, 3)):
+        launch()
+    ctx.check()
+
+    # ---- timed region: exactly K steps, device-timed on the launching stream
+    barrier()
+    with ClockSampler(local_rank) as clk:
+        if flush is None:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(args.steps):
+                launch()
+            e1.record()
+            torch.cuda.synchronize()
+            total_s = e0.elapsed_time(e1) * 1e-3
+        else:
+            total_s = float(sum(per_launch_times(ctx, p, dev, args.steps, flush)))
+    barrier()
+    ctx.check()
+    plan = ctx.last_plan()
+
+    # ---- end to end: host buffers in, host result out, every step
+    hA, hB, hBias, hR = pinned(p.A), pinned(p.B), pinned(p.bias), pinned(p.R if p.beta != 0 else None)
+    hD = torch.empty((p.batch, p.M, p.N), dtype=torch.int16).pin_memory()
+    e2e_call = lambda: ctx.gemm_epilogue_host(hA, hB, hBias, hR, hD, p.M, p.N, p.K, p.batch, p.alpha, p.beta, p.act)
+    for _ in range(3):
+        e2e_call()
+    e2e_steps = max(1, min(args.steps, 20))
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_call()
+    e1.record()
+    torch.cuda.synchronize()
+    e2e_s = e0.elapsed_time(e1) * 1e-3
+    barrier()
+    h2d = p.A.nbytes + p.B.nbytes + (p.bias.nbytes if p.bias is not None else 0) + (p.R.nbytes if hR is not None else 0)
+    d2h = hD.numel() * 2
+
+    if world > 1:
+        t = torch.tensor([total_s, e2e_s], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_s, e2e_s = float(t[0]), float(t[1])
+
+    value = world * p.flops * args.steps / total_s / 1e12
+    e2e_value = world * p.flops * e2e_steps / e2e_s / 1e12
+    per_launch_s = total_s / args.steps
+    bound = BOUND[args.config]
+    if bound == "hbm":
+        achieved, peak, runit = p.algorithmic_bytes / per_launch_s / 1e9, peaks["hbm_gbs"], "GB/s"
+    else:
+        achieved, peak, runit = p.flops / per_launch_s / 1e12, peaks["bf16_tflops"], "TFLOP/s"
+    roofline = {"bound": "hbm" if bound == "hbm" else "tensor", "achieved": achieved, "peak": peak, "unit": runit,
+                "frac": achieved / peak, "traffic": NCU_DRAM_TRAFFIC.get(args.config),
+                "peak_kind": f"burst, of {peaks['source']}", "frac_of_nominal": (achieved / 2250.0) if runit == "TFLOP/s" else (achieved / 8000.0),
+                "algorithmic_bytes": p.algorithmic_bytes, "flops": p.flops, "us_per_launch": per_launch_s * 1e6}
+
+    if rank != 0:
+        dist.destroy_process_group()
+        return
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": per_launch_s * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": describe(p), "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+                       "l2": "inputs larger than L2, launches back to back" if flush is None else
+                             "L2 flushed (252 MiB write) before every timed launch",
+                       "plan": plan},
+            "clocks": clk.summary(), "roofline": roofline,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                    "steps": e2e_steps, "ms_per_step": e2e_s / e2e_steps * 1e3},
+            "gpu_launches": args.steps}
+    if world == 1:
+        secs = 12.0
+        nrows = rows_for_seconds(p, secs)
+        dt, fl, n = oracle_sample(p, nrows)
+        line["cpu_baseline"] = {"value": fl / dt / 1e12, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                "sample": f"{n} of {p.batch * p.M} output rows (all N columns, full K) in {dt:.1f} s; "
+                                          f"host has {os.cpu_count()} cores, the oracle uses 1"}
+        if not args.no_table:
+            line["workloads"] = workload_table(ctx, device, peaks, W.CONFIG_ORDER)
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", default=DEFAULT_CONFIG, choices=W.CONFIG_ORDER)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-table", action="store_true", help="skip the five-workload table")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

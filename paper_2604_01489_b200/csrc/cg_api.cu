@@ -54,7 +54,7 @@ struct cg_context {
   int last_status = CG_OK;
   char last_msg[256] = {0};
   long long wait_limit = 4000000000ll;   // about two seconds of SM clocks
-  int max_pairs = 0;                     // co-resident CTA pairs, filled lazily per kernel
+  int test_starve = 0;                   // test hook (CG_TEST_STARVE): see KernelParams::test_starve
   StagingBuf sA, sB, sBias, sR, sD;
   std::mutex mu;
 };
@@ -280,6 +280,7 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   p.tickets = h->tickets;
   p.status = h->status;
   p.wait_limit = h->wait_limit;
+  p.test_starve = h->test_starve;
 
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof cfg);
@@ -365,6 +366,7 @@ int cg_create(cg_handle_t* out, int device, size_t workspace_bytes) {
     const long long v = atoll(w);
     if (v > 0) h->wait_limit = v;
   }
+  if (const char* w = getenv("CG_TEST_STARVE")) h->test_starve = atoi(w) != 0;
   *out = h;
   return CG_OK;
 }

@@ -71,6 +71,7 @@ struct KernelParams {
   int* tickets;           // [num_tiles * 4], zero between launches
   int* status;
   long long wait_limit;   // clock cycles before a wait gives up
+  int test_starve;        // test hook: the producer withholds the first A load, so `full[0]` never completes
 };
 
 template <int BN, int CG, bool B_KMAJOR>
@@ -292,60 +293,72 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       WorkIter wi(p, worker);
       Segment s;
       bool ok = true;
-      uint32_t filled_mask = 0, filled_parity = 0;   // stages with a load in flight and the phase it completes
+      long long issued = 0;                        // k-blocks handed to the TMA unit so far
+      const uint32_t full0 = ptx::smem_u32(&ctrl->full[0]);
+      const uint32_t empty0 = ptx::smem_u32(&ctrl->empty[0]);
+      const uint32_t full0_leader = (CG == 2) ? ptx::mapa(full0, 0) : full0;
       while (ok && wi.next(s)) {
         int b, mt, nt;
         decode_tile(p, s.tile, b, mt, nt);
         const int m0 = mt * (BM * CG) + static_cast<int>(cta_rank) * BM;
         const int n0 = nt * BN + static_cast<int>(cta_rank) * C::BN_CTA * (CG - 1);
         for (int kb = s.kb0; kb < s.kb1; ++kb) {
-          if (!wait_bar(ptx::smem_u32(&ctrl->empty[stage]), phase ^ 1u, ctrl, p)) { ok = false; break; }
-          const uint32_t full_local = ptx::smem_u32(&ctrl->full[stage]);
+          if (!wait_bar(empty0 + stage * 8, phase ^ 1u, ctrl, p)) { ok = false; break; }
           const uint32_t a_dst = ring_addr + stage * C::STAGE_BYTES;
           const uint32_t b_dst = a_dst + C::A_BYTES;
+          const int k0 = kb * BK;
           if constexpr (CG == 1) {
-            ptx::mbar_arrive_expect_tx(full_local, C::STAGE_BYTES);
-            ptx::tma_load_3d(a_dst, &tmA, full_local, kb * BK, m0, b);
+            const uint32_t bar = full0 + stage * 8;
+            ptx::mbar_arrive_expect_tx(bar, C::STAGE_BYTES);
+            if (!(p.test_starve && issued == 0)) ptx::tma_load_3d(a_dst, &tmA, bar, k0, m0, b);
             if constexpr (B_KMAJOR) {
-              ptx::tma_load_3d(b_dst, &tmB, full_local, kb * BK, n0, b);
+              ptx::tma_load_3d(b_dst, &tmB, bar, k0, n0, b);
             } else {
 #pragma unroll
               for (int j = 0; j < C::BN_CTA / 64; ++j)
-                ptx::tma_load_3d(b_dst + j * (64 * BK * 2), &tmB, full_local, n0 + j * 64, kb * BK, b);
+                ptx::tma_load_3d(b_dst + j * (64 * BK * 2), &tmB, bar, n0 + j * 64, k0, b);
             }
           } else {
             // both CTAs' bytes are counted on the leader's barrier
-            if (cta_rank == 0) ptx::mbar_arrive_expect_tx(full_local, 2 * C::STAGE_BYTES);
-            const uint32_t full_leader = ptx::mapa(full_local, 0);
-            ptx::tma_load_3d_pair(a_dst, &tmA, full_leader, kb * BK, m0, b);
+            if (cta_rank == 0) ptx::mbar_arrive_expect_tx(full0 + stage * 8, 2 * C::STAGE_BYTES);
+            const uint32_t bar = full0_leader + stage * 8;
+            if (!(p.test_starve && issued == 0)) ptx::tma_load_3d_pair(a_dst, &tmA, bar, k0, m0, b);
             if constexpr (B_KMAJOR) {
-              ptx::tma_load_3d_pair(b_dst, &tmB, full_leader, kb * BK, n0, b);
+              ptx::tma_load_3d_pair(b_dst, &tmB, bar, k0, n0, b);
             } else {
 #pragma unroll
               for (int j = 0; j < C::BN_CTA / 64; ++j)
-                ptx::tma_load_3d_pair(b_dst + j * (64 * BK * 2), &tmB, full_leader, n0 + j * 64, kb * BK, b);
+                ptx::tma_load_3d_pair(b_dst + j * (64 * BK * 2), &tmB, bar, n0 + j * 64, k0, b);
             }
           }
-          filled_mask |= 1u << stage;
-          filled_parity = (filled_parity & ~(1u << stage)) | (phase << stage);
+          ++issued;
           if (++stage == stages) { stage = 0; phase ^= 1u; }
         }
       }
       if (!ok || *reinterpret_cast<volatile int*>(&ctrl->abort)) {
-        // abort path: let this CTA's own copies land before shared memory is given up
+        // abort path: let the copies still in flight land before shared memory is given up.
+        // The leader can watch its `full` barriers; either CTA also sits out a fixed settle
+        // time that is far longer than any copy takes.
+        constexpr long long DRAIN_LIMIT = 1ll << 27;
         if (CG == 1 || cta_rank == 0) {
-          for (int s2 = 0; s2 < stages; ++s2)
-            if (filled_mask & (1u << s2)) {
-              const long long t0 = clock64();
-              while (!ptx::mbar_try_wait(ptx::smem_u32(&ctrl->full[s2]), (filled_parity >> s2) & 1u))
-                if (clock64() - t0 > p.wait_limit) break;
-            }
+          long long i = issued - stages;
+          if (i < 0) i = 0;
+          if (p.test_starve && i == 0) i = 1;      // the withheld load never completes its barrier
+          for (; i < issued; ++i) {
+            const long long t0 = clock64();
+            while (!ptx::mbar_try_wait(full0 + static_cast<uint32_t>(i % stages) * 8, static_cast<uint32_t>((i / stages) & 1)))
+              if (clock64() - t0 > DRAIN_LIMIT) break;
+          }
         }
+        const long long t1 = clock64();
+        while (clock64() - t1 < 100000) {}
       }
     }
     __syncwarp();
   } else if (warp == 1) {
     // ================================================================ MMA issuer
+    // One thread feeds the tensor pipe, so its instruction count per k-block is what bounds
+    // small tiles: descriptor words are precomputed and only their low (address) half moves.
     if (lane == 0 && (CG == 1 || cta_rank == 0)) {
       int stage = 0;
       uint32_t phase = 0;
@@ -354,33 +367,45 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       WorkIter wi(p, worker);
       Segment s;
       bool ok = true;
+      // descriptor = {lo: start address >> 4 | LBO >> 4 << 16, hi: SBO >> 4 | version | swizzle}
+      const uint64_t a_desc0 = ptx::smem_desc_sw128(ring_addr, 16, 8 * 128);
+      const uint64_t b_desc0 = B_KMAJOR ? ptx::smem_desc_sw128(ring_addr + C::A_BYTES, 16, 8 * 128)
+                                        : ptx::smem_desc_sw128(ring_addr + C::A_BYTES, 64 * BK * 2, 8 * 128);
+      const uint32_t desc_hi = static_cast<uint32_t>(a_desc0 >> 32);      // same for A and B
+      const uint32_t a_lo0 = static_cast<uint32_t>(a_desc0), b_lo0 = static_cast<uint32_t>(b_desc0);
+      constexpr uint32_t STAGE_STEP = C::STAGE_BYTES >> 4;
+      constexpr uint32_t A_KSTEP = (UMMA_K * 2) >> 4;                     // +32 B inside the swizzle row
+      constexpr uint32_t B_KSTEP = B_KMAJOR ? ((UMMA_K * 2) >> 4) : ((UMMA_K * 128) >> 4);   // or +16 k-rows
+      const uint32_t full0 = ptx::smem_u32(&ctrl->full[0]);
+      const uint32_t empty0 = ptx::smem_u32(&ctrl->empty[0]);
+      const uint32_t empty0_peer = (CG == 2) ? ptx::mapa(empty0, 1) : 0u;
+      const int last_kb = p.k_blocks - 1;
+      int tail_nk = (p.K - last_kb * BK + UMMA_K - 1) / UMMA_K;           // 16-wide steps of the last k-block
+      if (tail_nk > BK / UMMA_K) tail_nk = BK / UMMA_K;
+      auto desc = [&](uint32_t lo) -> uint64_t { return (static_cast<uint64_t>(desc_hi) << 32) | lo; };
       while (ok && wi.next(s)) {
         if (!wait_bar(ptx::smem_u32(&ctrl->acc_empty[acc]), acc_phase ^ 1u, ctrl, p)) { ok = false; break; }
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
+        uint32_t accumulate = 0;
         for (int kb = s.kb0; kb < s.kb1; ++kb) {
-          if (!wait_bar(ptx::smem_u32(&ctrl->full[stage]), phase, ctrl, p)) { ok = false; break; }
+          if (!wait_bar(full0 + stage * 8, phase, ctrl, p)) { ok = false; break; }
           ptx::tc_fence_after();
-          const uint32_t a_addr = ring_addr + stage * C::STAGE_BYTES;
-          const uint32_t b_addr = a_addr + C::A_BYTES;
-          int nk = (p.K - kb * BK + UMMA_K - 1) / UMMA_K;     // skip 16-wide steps that are all padding
-          if (nk > BK / UMMA_K) nk = BK / UMMA_K;
-          for (int k = 0; k < nk; ++k) {
-            // A, K-major: +16 elements along K = +32 bytes inside the 128-byte swizzle row
-            const uint64_t a_desc = ptx::smem_desc_sw128(a_addr + k * (UMMA_K * 2), 16, 8 * 128);
-            uint64_t b_desc;
-            if constexpr (B_KMAJOR) {
-              b_desc = ptx::smem_desc_sw128(b_addr + k * (UMMA_K * 2), 16, 8 * 128);
-            } else {
-              // B, N-major: rows are k, 128 B = 64 n; +16 k = two 8-row groups = +2048 bytes;
-              // 64-column blocks are whole TMA boxes, 64*64*2 bytes apart
-              b_desc = ptx::smem_desc_sw128(b_addr + k * (UMMA_K * 128), 64 * BK * 2, 8 * 128);
-            }
-            ptx::mma_f16<CG>(d_tmem, a_desc, b_desc, C::IDESC, (kb > s.kb0 || k > 0) ? 1u : 0u);
+          const uint32_t a_lo = a_lo0 + stage * STAGE_STEP;
+          const uint32_t b_lo = b_lo0 + stage * STAGE_STEP;
+          if (kb != last_kb || tail_nk == BK / UMMA_K) {
+            ptx::mma_f16<CG>(d_tmem, desc(a_lo), desc(b_lo), C::IDESC, accumulate);
+            ptx::mma_f16<CG>(d_tmem, desc(a_lo + A_KSTEP), desc(b_lo + B_KSTEP), C::IDESC, 1u);
+            ptx::mma_f16<CG>(d_tmem, desc(a_lo + 2 * A_KSTEP), desc(b_lo + 2 * B_KSTEP), C::IDESC, 1u);
+            ptx::mma_f16<CG>(d_tmem, desc(a_lo + 3 * A_KSTEP), desc(b_lo + 3 * B_KSTEP), C::IDESC, 1u);
+          } else {
+            for (int k = 0; k < tail_nk; ++k)     // K tail: skip 16-wide steps that are all padding
+              ptx::mma_f16<CG>(d_tmem, desc(a_lo + k * A_KSTEP), desc(b_lo + k * B_KSTEP), C::IDESC,
+                               (k > 0) ? 1u : accumulate);
           }
-          const uint32_t empty_local = ptx::smem_u32(&ctrl->empty[stage]);
-          ptx::tc_commit<CG>(empty_local);
-          if constexpr (CG == 2) ptx::tc_commit<CG>(ptx::mapa(empty_local, 1));
+          accumulate = 1u;
+          ptx::tc_commit<CG>(empty0 + stage * 8);
+          if constexpr (CG == 2) ptx::tc_commit<CG>(empty0_peer + stage * 8);
           if (++stage == stages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
@@ -395,7 +420,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         ptx::tc_commit<CG>(ptx::smem_u32(&ctrl->drain));
         const long long t0 = clock64();
         while (!ptx::mbar_try_wait(ptx::smem_u32(&ctrl->drain), 0))
-          if (clock64() - t0 > p.wait_limit) break;
+          if (clock64() - t0 > (1ll << 27)) break;
       }
     }
     __syncwarp();
