@@ -246,7 +246,7 @@ def run_ours(args):
     if footprint <= 2 * L2_BYTES:                  # inputs could sit in L2: flush between timed launches
         flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=device)
 
-    for _ in range(max(args.warmup, 3)):
+    for _ in range(args.warmup if args.kernel_only else max(args.warmup, 3)):
         launch()
     ctx.check()
 
@@ -268,23 +268,24 @@ def run_ours(args):
     plan = ctx.last_plan()
 
     # ---- end to end: host buffers in, host result out, every step
-    hA, hB, hBias, hR = pinned(p.A), pinned(p.B), pinned(p.bias), pinned(p.R if p.beta != 0 else None)
-    hD = torch.empty((p.batch, p.M, p.N), dtype=torch.int16).pin_memory()
-    e2e_call = lambda: ctx.gemm_epilogue_host(hA, hB, hBias, hR, hD, p.M, p.N, p.K, p.batch, p.alpha, p.beta, p.act)
-    for _ in range(3):
-        e2e_call()
-    e2e_steps = max(1, min(args.steps, 20))
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(e2e_steps):
-        e2e_call()
-    e1.record()
-    torch.cuda.synchronize()
-    e2e_s = e0.elapsed_time(e1) * 1e-3
-    barrier()
-    h2d = p.A.nbytes + p.B.nbytes + (p.bias.nbytes if p.bias is not None else 0) + (p.R.nbytes if hR is not None else 0)
-    d2h = hD.numel() * 2
+    e2e_steps, e2e_s, h2d, d2h = max(1, min(args.steps, 20)), float("nan"), 0, 0
+    if not args.kernel_only:
+        hA, hB, hBias, hR = pinned(p.A), pinned(p.B), pinned(p.bias), pinned(p.R if p.beta != 0 else None)
+        hD = torch.empty((p.batch, p.M, p.N), dtype=torch.int16).pin_memory()
+        e2e_call = lambda: ctx.gemm_epilogue_host(hA, hB, hBias, hR, hD, p.M, p.N, p.K, p.batch, p.alpha, p.beta, p.act)
+        for _ in range(3):
+            e2e_call()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(e2e_steps):
+            e2e_call()
+        e1.record()
+        torch.cuda.synchronize()
+        e2e_s = e0.elapsed_time(e1) * 1e-3
+        barrier()
+        h2d = p.A.nbytes + p.B.nbytes + (p.bias.nbytes if p.bias is not None else 0) + (p.R.nbytes if hR is not None else 0)
+        d2h = hD.numel() * 2
 
     if world > 1:
         t = torch.tensor([total_s, e2e_s], dtype=torch.float64, device=device)
@@ -318,7 +319,9 @@ def run_ours(args):
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                     "steps": e2e_steps, "ms_per_step": e2e_s / e2e_steps * 1e3},
             "gpu_launches": args.steps}
-    if world == 1:
+    if args.kernel_only:
+        line["e2e"] = None
+    if world == 1 and not args.kernel_only:
         secs = 12.0
         nrows = rows_for_seconds(p, secs)
         dt, fl, n = oracle_sample(p, nrows)
@@ -340,6 +343,8 @@ def main():
     ap.add_argument("--config", default=DEFAULT_CONFIG, choices=W.CONFIG_ORDER)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-table", action="store_true", help="skip the five-workload table")
+    ap.add_argument("--kernel-only", action="store_true",
+                    help="only the device-timed region (for profiler runs): no e2e, no CPU baseline, no table")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
