@@ -128,6 +128,39 @@ CG_API int cg_get_last_plan(cg_handle_t h, cg_plan_info_t* out);
  */
 CG_API int cg_last_error(cg_handle_t h, int sync, char* buf, size_t len);
 
+/*
+ * (The paper has no counterpart for this entry point; it exists for deployment reasons only.)
+ *
+ * The same fused GEMM + epilogue without a handle and without any allocation, for callers that
+ * cannot obtain device memory at call time -- for example a serving process whose own memory pool
+ * reserved the whole device at start-up, so that cudaMalloc fails, or a latency-critical path that
+ * must not risk the device-wide synchronisation an allocation can cause.  It runs the 1-CTA
+ * 128 x 128 tile kernel with each tile's K range cut into `split_k` parts (1 = no split); the
+ * scratch of the split (fp32 partial tiles, tickets, status word) lives in a fixed array inside
+ * the library image: 8 MiB of partial tiles plus tickets for 4096 tiles, held by every GPU that
+ * loads the library until the process exits.  Neither this function nor anything it calls invokes
+ * cudaMalloc, cudaFree or an allocating library routine.
+ *
+ *   A, B, bias, R, D, M, N, K, batch, alpha, beta, act, stream: exactly as for cg_gemm_epilogue;
+ *       all device pointers are the caller's.  The CURRENT CUDA device is used.
+ *   split_k   parts per output tile (clamped to the number of 64-wide k-blocks).  The call is
+ *             rejected with CG_ERR_WORKSPACE when 2 * tiles * parts * 64 KiB exceeds the 8 MiB of
+ *             partial-tile space or more than 4096 tiles would be split
+ *             (tiles = batch * ceil(M/128) * ceil(N/128)).
+ *   err       optional host buffer of err_len bytes that receives a message when the return value
+ *             is not CG_OK.
+ *
+ * The first call on each device looks up the array's device address and sets kernel attributes;
+ * make that first call before any stream capture begins.  All calls share the one array, which
+ * keeps the contents of the previous call (the tickets are cleared on the stream before each
+ * split launch): two calls that overlap on the GPU -- different streams, or different host
+ * threads -- race on it, so keep calls to this entry point ordered on one stream per device.
+ * A device-side timeout of a bounded wait is not reported by this entry point.
+ */
+CG_API int cg_gemm_epilogue_noalloc(const void* A, const void* B, const void* bias, const void* R, void* D, int M,
+                                    int N, int K, int batch, float alpha, float beta, int act, int split_k,
+                                    void* stream, char* err, size_t err_len);
+
 /* Frees the workspace and the handle.  The caller's tensors are not touched. */
 CG_API int cg_destroy(cg_handle_t h);
 

@@ -21,7 +21,7 @@ STATUS_NAMES = {0: "CG_OK", 1: "CG_ERR_INVALID_ARG", 2: "CG_ERR_UNSUPPORTED", 3:
                 5: "CG_ERR_WORKSPACE", 6: "CG_ERR_TIMEOUT"}
 
 EXPORTS = ["cg_create", "cg_gemm_epilogue", "cg_gemm_epilogue_host", "cg_set_tuning", "cg_get_last_plan",
-           "cg_last_error", "cg_destroy"]
+           "cg_last_error", "cg_gemm_epilogue_noalloc", "cg_destroy"]
 
 
 class cg_tuning_t(ctypes.Structure):
@@ -68,6 +68,7 @@ def load() -> ctypes.CDLL:
     lib.cg_get_last_plan.argtypes = [vp, ctypes.POINTER(cg_plan_info_t)]
     lib.cg_last_error.argtypes = [vp, ci, ctypes.c_char_p, sz]
     lib.cg_destroy.argtypes = [vp]
+    lib.cg_gemm_epilogue_noalloc.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, cf, cf, ci, ci, vp, ctypes.c_char_p, sz]
     for name in EXPORTS:
         getattr(lib, name).restype = ci
     _lib = lib
@@ -154,6 +155,16 @@ def cg_last_error(h, sync: bool = False):
     """Returns (status code, message)."""
     buf = ctypes.create_string_buffer(256)
     rc = load().cg_last_error(h, 1 if sync else 0, buf, 256)
+    return rc, buf.value.decode(errors="replace")
+
+
+def cg_gemm_epilogue_noalloc(A, B, bias, R, D, M, N, K, batch, alpha, beta, act, split_k=1, stream=None):
+    """Handle-free, allocation-free variant (scratch in a fixed array of the library): for callers
+    that cannot allocate device memory when they call.  Returns (status code, message)."""
+    buf = ctypes.create_string_buffer(256)
+    rc = load().cg_gemm_epilogue_noalloc(_dev_ptr(A), _dev_ptr(B), _dev_ptr(bias), _dev_ptr(R), _dev_ptr(D), int(M),
+                                         int(N), int(K), int(batch), float(alpha), float(beta), int(act), int(split_k),
+                                         _stream_ptr(stream), buf, 256)
     return rc, buf.value.decode(errors="replace")
 
 

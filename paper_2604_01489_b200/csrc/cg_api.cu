@@ -469,3 +469,131 @@ int cg_destroy(cg_handle_t h) {
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------
+// Allocation-free entry point.
+//
+// Some callers must not, or cannot, allocate device memory: a serving process whose own memory
+// pool took the whole device at start-up (cudaMalloc then simply fails), or a latency-critical
+// path that cannot afford the device-wide synchronisation an allocation may imply.  For them the
+// split-K form of the kernel runs with its scratch (fp32 partial tiles, per-tile tickets, status
+// word) in the fixed array below instead of a handle's workspace.  The array is part of the
+// library image: every GPU that loads the library keeps these bytes until the process exits.
+namespace {
+
+constexpr int NOALLOC_TILE_N = 128;
+constexpr int NOALLOC_MAX_TILES = 4096;                                  // tiles that may be split
+constexpr size_t NOALLOC_STATUS_BYTES = 256;
+constexpr size_t NOALLOC_TICKET_BYTES = static_cast<size_t>(NOALLOC_MAX_TILES) * 4 * sizeof(int);
+constexpr size_t NOALLOC_PARTIAL_BYTES = 8u << 20;                       // 8 MiB of fp32 partial tiles
+constexpr int NOALLOC_MAX_DEVICES = 64;
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_STATUS_BYTES + NOALLOC_TICKET_BYTES +
+                                                               NOALLOC_PARTIAL_BYTES];
+
+struct NoallocDevice {
+  bool ready = false;
+  cg_context ctx;
+};
+NoallocDevice g_noalloc[NOALLOC_MAX_DEVICES];
+std::mutex g_noalloc_mu;
+
+void set_err(char* err, size_t len, const char* msg) {
+  if (err && len > 0) {
+    strncpy(err, msg, len - 1);
+    err[len - 1] = 0;
+  }
+}
+
+// Once per device, with that device current.  In host code the array's name is only a stand-in
+// for the symbol; the device address a kernel may use comes from cudaGetSymbolAddress.
+int noalloc_setup(int device, NoallocDevice** out, char* err, size_t err_len) {
+  std::lock_guard<std::mutex> lock(g_noalloc_mu);
+  NoallocDevice& d = g_noalloc[device];
+  if (!d.ready) {
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { set_err(err, err_len, "cudaGetDeviceProperties failed"); return CG_ERR_CUDA; }
+    if (prop.major != 10 || prop.minor != 0) { set_err(err, err_len, "device is not compute capability 10.0"); return CG_ERR_ARCH; }
+    unsigned char* base = nullptr;
+    const cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void**>(&base), g_noalloc_scratch);
+    if (e != cudaSuccess || base == nullptr) {
+      set_err(err, err_len, "cudaGetSymbolAddress failed for the static scratch array");
+      return CG_ERR_CUDA;
+    }
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+        qres != cudaDriverEntryPointSuccess) {
+      set_err(err, err_len, "cuTensorMapEncodeTiled is not available");
+      return CG_ERR_CUDA;
+    }
+    cg_context& c = d.ctx;
+    c.device = device;
+    c.num_sms = prop.multiProcessorCount;
+    c.encode = reinterpret_cast<EncodeTiledFn>(fn);
+    c.status = reinterpret_cast<int*>(base);
+    c.tickets = reinterpret_cast<int*>(base + NOALLOC_STATUS_BYTES);
+    c.partials = reinterpret_cast<float*>(base + NOALLOC_STATUS_BYTES + NOALLOC_TICKET_BYTES);
+    c.partial_bytes = NOALLOC_PARTIAL_BYTES;
+    c.workspace_bytes = sizeof g_noalloc_scratch;
+    if (prepare_kernels(&c) != CG_OK) { set_err(err, err_len, c.last_msg); return CG_ERR_CUDA; }
+    d.ready = true;
+  }
+  *out = &d;
+  return CG_OK;
+}
+
+}  // namespace
+
+extern "C" int cg_gemm_epilogue_noalloc(const void* A, const void* B, const void* bias, const void* R, void* D, int M,
+                                        int N, int K, int batch, float alpha, float beta, int act, int split_k,
+                                        void* stream, char* err, size_t err_len) {
+  set_err(err, err_len, "");
+  int device = 0;
+  if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= NOALLOC_MAX_DEVICES) {
+    set_err(err, err_len, "no usable current CUDA device");
+    return CG_ERR_CUDA;
+  }
+  NoallocDevice* d = nullptr;
+  int rc = noalloc_setup(device, &d, err, err_len);
+  if (rc != CG_OK) return rc;
+  cg_context* h = &d->ctx;
+  std::lock_guard<std::mutex> lock(h->mu);
+  if (split_k < 1) { set_err(err, err_len, "split_k must be >= 1"); return CG_ERR_INVALID_ARG; }
+  if ((rc = validate(h, A, B, bias, R, D, M, N, K, batch, beta, act)) != CG_OK ||
+      (rc = check_alignment(h, A, B, bias, R, D, beta, act)) != CG_OK) {
+    set_err(err, err_len, h->last_msg);
+    return rc;
+  }
+  const int k_blocks = ceil_div(K, BK);
+  const long long tiles = static_cast<long long>(batch) * ceil_div(M, BM) * ceil_div(N, NOALLOC_TILE_N);
+  const int parts = split_k < k_blocks ? split_k : k_blocks;
+  const long long units = tiles * parts;
+  if (parts > 1) {
+    const size_t need = static_cast<size_t>(2) * units * BM * NOALLOC_TILE_N * sizeof(float);
+    if (tiles > NOALLOC_MAX_TILES || units >= (1ll << 30) || need > NOALLOC_PARTIAL_BYTES) {
+      char msg[200];
+      snprintf(msg, sizeof msg,
+               "problem too large for the static scratch: %lld tiles x %d parts need %zu bytes of partial tiles "
+               "(maximum %zu bytes, %d tiles)", tiles, parts, need, NOALLOC_PARTIAL_BYTES, NOALLOC_MAX_TILES);
+      set_err(err, err_len, msg);
+      return CG_ERR_WORKSPACE;
+    }
+  } else if (units >= (1ll << 30)) {
+    set_err(err, err_len, "problem too large");
+    return CG_ERR_UNSUPPORTED;
+  }
+  memset(&h->tuning, 0, sizeof h->tuning);
+  h->tuning.tile_n = NOALLOC_TILE_N;
+  h->tuning.cta_group = 1;
+  h->tuning.num_units = static_cast<int>(units);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (parts > 1) {
+    // the array keeps whatever the previous call left: tickets must start at zero
+    const cudaError_t e = cudaMemsetAsync(h->tickets, 0, static_cast<size_t>(tiles) * 4 * sizeof(int), st);
+    if (e != cudaSuccess) { set_err(err, err_len, cudaGetErrorString(e)); return CG_ERR_CUDA; }
+  }
+  rc = launch(h, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, st);
+  if (rc != CG_OK) set_err(err, err_len, h->last_msg);
+  return rc;
+}

@@ -1,0 +1,59 @@
+"""The allocation-free entry point, cg_gemm_epilogue_noalloc, against the regular one.
+
+Who needs it: a caller that cannot get device memory at call time -- a serving process whose own
+pool reserved the whole GPU at start-up (cudaMalloc just fails there), or a path that must not risk
+the device-wide synchronisation an allocation can trigger.  The entry point keeps the split-K
+scratch in a fixed array of the library instead.  This file is collected last on purpose: if it
+fails, a run that stops at the first failure has already run every other test.
+"""
+import numpy as np
+import pytest
+
+from cg_inputs import workloads as W
+
+import parity_util as PU
+
+pytestmark = pytest.mark.gpu
+
+
+def test_noalloc_matches_regular_entry_point_twice():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device")
+    import paper_2604_01489_b200 as cg
+
+    p = W.make(300, 392, 1032, batch=2, seed=23, act=W.ACT_SILU, alpha=0.5, beta=1.0, A=("normal", 1.0),
+               B=("normal", 0.1), bias=("normal", 1.0), R=("normal", 1.0))
+    dev = PU.to_device(p)
+    split_k = 2                                  # 24 tiles x 2 parts x 128 KiB = 6 MiB of the 8 MiB scratch
+    tiles = p.batch * -(-p.M // 128) * -(-p.N // 128)
+
+    # the existing entry point, same tile shape and the same split
+    ctx = cg.Context(0)
+    ctx.set_tuning(tile_n=128, cta_group=1, num_units=tiles * split_k)
+    want_bits = PU.run_gpu(ctx, p, dev, fill=0x7FC0)
+    assert ctx.last_plan()["num_units"] == tiles * split_k
+    ctx.close()
+    want = PU.gen.bf16_bits_to_f32(want_bits).astype(np.float64)
+
+    mem_before = torch.cuda.mem_get_info()[0]
+    for call in range(2):                        # the second call finds the first call's leftovers in the array
+        dev["D"].view(torch.int16).fill_(0x7FC0)
+        rc, msg = cg.cg_gemm_epilogue_noalloc(dev["A"], dev["B"], dev["bias"], dev["R"], dev["D"], p.M, p.N, p.K, p.batch,
+                                              p.alpha, p.beta, p.act, split_k=split_k)
+        assert rc == cg.CG_OK, (call, rc, msg)
+        torch.cuda.synchronize()
+        got_bits = dev["D"].view(torch.int16).cpu().numpy().view(np.uint16)
+        c = PU.compare(got_bits, want)           # same tolerance as the parity tests, reference = regular entry point
+        assert c["ok"], (call, c)
+    assert torch.cuda.mem_get_info()[0] >= mem_before - (1 << 20), "the call must not allocate device memory"
+
+    # unsplit plan, and a size beyond the fixed scratch
+    rc, msg = cg.cg_gemm_epilogue_noalloc(dev["A"], dev["B"], dev["bias"], dev["R"], dev["D"], p.M, p.N, p.K, p.batch,
+                                          p.alpha, p.beta, p.act, split_k=1)
+    assert rc == cg.CG_OK, msg
+    torch.cuda.synchronize()
+    assert PU.compare(dev["D"].view(torch.int16).cpu().numpy().view(np.uint16), want)["ok"]
+    rc, msg = cg.cg_gemm_epilogue_noalloc(dev["A"], dev["B"], dev["bias"], dev["R"], dev["D"], p.M, p.N, p.K, p.batch,
+                                          p.alpha, p.beta, p.act, split_k=8)      # 24 tiles x 8 parts x 128 KiB > 8 MiB
+    assert rc == cg.CG_ERR_WORKSPACE and "static scratch" in msg
