@@ -98,7 +98,7 @@ CG_API int cg_gemm_epilogue_host(cg_handle_t h, const void* A, const void* B, co
  * A non-zero field forces that choice for the following calls on this handle.
  */
 typedef struct cg_tuning {
-  int tile_n;    /* 64, 128 or 256: accumulator tile width                                  */
+  int tile_n;    /* 64, 128, 256, or 512 (CTA pairs only): accumulator tile width           */
   int cta_group; /* 1 = one CTA per 128-row tile, 2 = CTA pair sharing a 256-row tile       */
   int num_units; /* number of contiguous k-block ranges the iteration space is cut into:
                     = number of tiles -> data-parallel, a multiple of it -> split-K,

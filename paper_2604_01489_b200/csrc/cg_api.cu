@@ -86,13 +86,14 @@ typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const CUtensorMap
 
 struct KernelEntry {
   KernelFn fn;
-  int stage_bytes, fixed_bytes, stages_max;
+  int stage_bytes, fixed_bytes, stages_max, threads, sub_cols;
 };
 
 template <int BN, int CGN, bool KM>
 KernelEntry entry() {
   using C = Cfg<BN, CGN, KM>;
-  return KernelEntry{gemm_epilogue_kernel<BN, CGN, KM>, C::STAGE_BYTES, C::FIXED_BYTES, C::STAGES_MAX};
+  return KernelEntry{gemm_epilogue_kernel<BN, CGN, KM>, C::STAGE_BYTES, C::FIXED_BYTES, C::STAGES_MAX, C::NUM_THREADS,
+                     C::SUB_COLS};
 }
 
 // index: [bn_idx (64,128,256)][cg-1][b_kmajor]
@@ -104,14 +105,15 @@ bool lookup(int bn, int cgn, bool km, KernelEntry* out) {
   } else if (cgn == 2) {
     if (bn == 128) { *out = km ? entry<128, 2, true>() : entry<128, 2, false>(); return true; }
     if (bn == 256) { *out = km ? entry<256, 2, true>() : entry<256, 2, false>(); return true; }
+    if (bn == 512) { *out = km ? entry<512, 2, true>() : entry<512, 2, false>(); return true; }
   }
   return false;
 }
 
 int prepare_kernels(cg_context* h) {
-  const int bns[3] = {64, 128, 256};
+  const int bns[4] = {64, 128, 256, 512};
   for (int cgn = 1; cgn <= 2; ++cgn)
-    for (int i = 0; i < 3; ++i)
+    for (int i = 0; i < 4; ++i)
       for (int km = 0; km < 2; ++km) {
         KernelEntry e;
         if (!lookup(bns[i], cgn, km != 0, &e)) continue;
@@ -160,6 +162,14 @@ int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, Plan
   if (bn == 0) {
     if (cgn == 2) {
       bn = (N >= 256) ? 256 : 128;
+      // The 512-wide pair tile fetches a quarter fewer bytes from L2 per flop (two MMAs share A),
+      // but has half as many tiles: take it when it does not cost wave efficiency.
+      if (N >= 512) {
+        const int pairs = sms / 2 > 0 ? sms / 2 : 1;
+        auto eff = [&](long long nt) { return static_cast<double>(nt) / (static_cast<double>((nt + pairs - 1) / pairs) * pairs); };
+        const long long t256 = tiles(2 * BM, 256), t512 = tiles(2 * BM, 512);
+        if (t512 >= 2 * pairs && eff(t512) >= eff(t256) - 0.03) bn = 512;
+      }
     } else {
       // widest tile that still gives every SM a tile; otherwise the narrowest
       bn = 64;
@@ -211,9 +221,10 @@ int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, Plan
   if (stages > e.stages_max) stages = e.stages_max;
   if (stages < 1) stages = 1;
   pl->stages = stages;
-  pl->smem = stages * e.stage_bytes + e.fixed_bytes;
+  pl->smem = stages * e.stage_bytes + e.fixed_bytes + 1024;     // layout + alignment slack, capped at the limit
+  if (pl->smem > SMEM_LIMIT) pl->smem = SMEM_LIMIT;
 
-  int gm = t.group_m > 0 ? t.group_m : 8;
+  int gm = t.group_m > 0 ? t.group_m : (bn == 512 ? 16 : 8);
   if (gm > pl->tiles_m) gm = pl->tiles_m;
   pl->group_m = gm;
   return CG_OK;
@@ -252,9 +263,8 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   lookup(pl.bn, pl.cg, b_kmajor, &e);
 
   CUtensorMap tmA, tmB, tmD;
-  const int bn_cta = pl.bn / pl.cg;
   if ((rc = make_map(h, &tmA, A, K, M, batch, BK, BM)) != CG_OK) return rc;
-  if (b_kmajor) rc = make_map(h, &tmB, B, K, N, batch, BK, bn_cta);
+  if (b_kmajor) rc = make_map(h, &tmB, B, K, N, batch, BK, e.sub_cols);
   else rc = make_map(h, &tmB, B, N, K, batch, 64, BK);
   if (rc != CG_OK) return rc;
   if ((rc = make_map(h, &tmD, D, N, M, batch, EPI_COLS, 32)) != CG_OK) return rc;
@@ -285,7 +295,7 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof cfg);
   cfg.gridDim = dim3(pl.grid, 1, 1);
-  cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+  cfg.blockDim = dim3(e.threads, 1, 1);
   cfg.dynamicSmemBytes = pl.smem;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
@@ -415,7 +425,7 @@ int cg_set_tuning(cg_handle_t h, const cg_tuning_t* t) {
     memset(&h->tuning, 0, sizeof h->tuning);
     return CG_OK;
   }
-  if ((t->tile_n != 0 && t->tile_n != 64 && t->tile_n != 128 && t->tile_n != 256) || t->cta_group < 0 ||
+  if ((t->tile_n != 0 && t->tile_n != 64 && t->tile_n != 128 && t->tile_n != 256 && t->tile_n != 512) || t->cta_group < 0 ||
       t->cta_group > 2 || t->num_units < 0 || t->stages < 0 || t->group_m < 0 || t->max_ctas < 0)
     return fail(h, CG_ERR_INVALID_ARG, "bad tuning values");
   h->tuning = *t;

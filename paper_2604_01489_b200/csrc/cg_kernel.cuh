@@ -25,6 +25,12 @@
 // 128 rows of A and half of the B columns, the leader CTA issues tcgen05.mma.cta_group::2,
 // each CTA's epilogue drains its own 128 accumulator rows.
 //
+// BN == 512 (CTA pairs only) is the wide form for large compute-bound problems: two N = 256 MMAs
+// per 16-wide k-step share one A operand, which cuts the bytes fetched from L2 per flop by a
+// quarter (the L2-to-SM path, not the tensor pipe, is what stalls the 256 x 256 form).  Its
+// accumulator fills all 512 TMEM columns, so it is single-buffered and eight epilogue warps
+// (two per TMEM lane quarter, half the columns each) drain it.
+//
 // Every wait is bounded: when a limit expires the CTA records CG_ERR_TIMEOUT in the status
 // word, raises a CTA-wide abort flag that all roles poll, and every role leaves its loop,
 // still frees tensor memory and returns.
@@ -39,18 +45,14 @@ namespace cg {
 constexpr int BM = 128;          // accumulator rows per CTA (TMEM lanes)
 constexpr int BK = 64;           // k-block: 64 bf16 = one 128-byte swizzle row
 constexpr int UMMA_K = 16;       // K of one tcgen05.mma for 16-bit inputs
-constexpr int NUM_THREADS = 192;
 constexpr int MAX_STAGES = 12;
 constexpr int SMEM_LIMIT = 232448;  // 227 KiB opt-in maximum per CTA
 constexpr int EPI_COLS = 64;        // columns per epilogue chunk (one 128-byte bf16 row)
 constexpr int EPI_BUF_BYTES = 32 * EPI_COLS * 2;   // one warp's staging buffer: 32 rows x 128 B
-constexpr int EPI_BUFS = 2;
-constexpr int EPI_BYTES = 4 * EPI_BUFS * EPI_BUF_BYTES;
-constexpr int BIAS_BYTES = 4 * EPI_COLS * 4;       // per warp: one chunk of fp32 bias
-constexpr int CTRL_BYTES = 512;
+constexpr int CTRL_BYTES = 256;
 
 enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU_TANH = 2, ACT_SILU = 3 };
-enum { STATUS_OK = 0, STATUS_TIMEOUT = 6 };
+enum { STATUS_OK = 0, STATUS_SMEM = 4, STATUS_TIMEOUT = 6 };
 
 struct KernelParams {
   int M, N, K, batch;
@@ -76,18 +78,34 @@ struct KernelParams {
 
 template <int BN, int CG, bool B_KMAJOR>
 struct Cfg {
-  static_assert(BN == 64 || BN == 128 || BN == 256, "tile width");
+  static_assert(BN == 64 || BN == 128 || BN == 256 || BN == 512, "tile width");
   static_assert(CG == 1 || CG == 2, "cta group");
-  static constexpr int BN_CTA = BN / CG;                 // B columns each CTA loads
+  static_assert(BN != 512 || CG == 2, "the 512-wide tile exists for CTA pairs only");
+  static constexpr int MMA_N = BN > 256 ? 256 : BN;      // N of one tcgen05.mma
+  static constexpr int NSUB = BN / MMA_N;                // MMAs per k-step that share the A operand
+  static constexpr int SUB_COLS = MMA_N / CG;            // B columns this CTA loads per sub-MMA
+  static constexpr int BN_CTA = NSUB * SUB_COLS;         // B columns this CTA loads per k-block
   static constexpr int A_BYTES = BM * BK * 2;
-  static constexpr int B_BYTES = BN_CTA * BK * 2;
+  static constexpr int SUB_B_BYTES = SUB_COLS * BK * 2;
+  static constexpr int B_BYTES = NSUB * SUB_B_BYTES;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int FIXED_BYTES = EPI_BYTES + BIAS_BYTES + CTRL_BYTES + 1024;  // + alignment slack
+  static constexpr int ACC_BUFS = (2 * BN <= 512) ? 2 : 1;   // accumulator buffers in TMEM
+  static constexpr int EPI_WARPS = (BN == 512) ? 8 : 4;
+  static constexpr int EPI_COL_GROUPS = EPI_WARPS / 4;       // warps per TMEM lane quarter
+  static constexpr int EPI_BUFS = (EPI_WARPS == 4) ? 2 : 1;  // staging buffers per warp
+  static constexpr int NUM_THREADS = 64 + 32 * EPI_WARPS;
+  static constexpr int EPI_BYTES = EPI_WARPS * EPI_BUFS * EPI_BUF_BYTES;
+  static constexpr int BIAS_BYTES = EPI_WARPS * EPI_COLS * 4;   // per warp: one chunk of fp32 bias
+  static constexpr int FIXED_BYTES = EPI_BYTES + BIAS_BYTES + CTRL_BYTES;
+  // Up to 1023 bytes go to aligning the ring; the kernel checks that what is left suffices.
   static constexpr int MAX_FIT = (SMEM_LIMIT - FIXED_BYTES) / STAGE_BYTES;
   static constexpr int STAGES_MAX = MAX_FIT < MAX_STAGES ? MAX_FIT : MAX_STAGES;
-  static constexpr int TMEM_COLS = 2 * BN <= 32 ? 32 : (2 * BN <= 64 ? 64 : (2 * BN <= 128 ? 128 : (2 * BN <= 256 ? 256 : 512)));
-  static constexpr uint32_t IDESC = ptx::instr_desc_bf16(BM * CG, BN, !B_KMAJOR);
-  static constexpr int smem_bytes(int stages) { return stages * STAGE_BYTES + FIXED_BYTES; }
+  static constexpr int TMEM_COLS = ACC_BUFS * BN <= 32 ? 32 : (ACC_BUFS * BN <= 64 ? 64 : (ACC_BUFS * BN <= 128 ? 128 : (ACC_BUFS * BN <= 256 ? 256 : 512)));
+  static constexpr uint32_t IDESC = ptx::instr_desc_bf16(BM * CG, MMA_N, !B_KMAJOR);
+  __host__ __device__ static constexpr int layout_bytes(int stages) { return stages * STAGE_BYTES + FIXED_BYTES; }
+  __host__ __device__ static constexpr int smem_bytes(int stages) {      // request: the layout plus alignment slack, capped at the limit
+    return layout_bytes(stages) + 1024 < SMEM_LIMIT ? layout_bytes(stages) + 1024 : SMEM_LIMIT;
+  }
 };
 
 struct Ctrl {
@@ -235,7 +253,7 @@ __device__ __forceinline__ void epilogue_chunk(const float (&acc)[EPI_COLS], con
 // ---------------------------------------------------------------- the kernel
 
 template <int BN, int CG, bool B_KMAJOR>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__((Cfg<BN, CG, B_KMAJOR>::NUM_THREADS), 1)
 gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                      const __grid_constant__ CUtensorMap tmD, const KernelParams p) {
   using C = Cfg<BN, CG, B_KMAJOR>;
@@ -247,8 +265,16 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   const int stages = p.stages;
   uint8_t* epi_ptr = smem + stages * C::STAGE_BYTES;
   const uint32_t epi_addr = ring_addr + stages * C::STAGE_BYTES;
-  float* bias_all = reinterpret_cast<float*>(epi_ptr + EPI_BYTES);
-  Ctrl* ctrl = reinterpret_cast<Ctrl*>(epi_ptr + EPI_BYTES + BIAS_BYTES);
+  float* bias_all = reinterpret_cast<float*>(epi_ptr + C::EPI_BYTES);
+  Ctrl* ctrl = reinterpret_cast<Ctrl*>(epi_ptr + C::EPI_BYTES + C::BIAS_BYTES);
+  {
+    uint32_t dyn_bytes;
+    asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn_bytes));
+    if (pad + static_cast<uint32_t>(C::layout_bytes(stages)) > dyn_bytes) {   // never expected: the ring would not fit
+      if (threadIdx.x == 0) atomicCAS(p.status, STATUS_OK, STATUS_SMEM);
+      return;
+    }
+  }
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -263,7 +289,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(ptx::smem_u32(&ctrl->acc_full[a]), 1);
-      ptx::mbar_init(ptx::smem_u32(&ctrl->acc_empty[a]), 4 * CG);   // one arrive per epilogue warp of the pair
+      ptx::mbar_init(ptx::smem_u32(&ctrl->acc_empty[a]), C::EPI_WARPS * CG);   // one arrive per epilogue warp of the pair
     }
     ptx::mbar_init(ptx::smem_u32(&ctrl->drain), 1);
     ctrl->abort = 0;
@@ -301,7 +327,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         int b, mt, nt;
         decode_tile(p, s.tile, b, mt, nt);
         const int m0 = mt * (BM * CG) + static_cast<int>(cta_rank) * BM;
-        const int n0 = nt * BN + static_cast<int>(cta_rank) * C::BN_CTA * (CG - 1);
+        const int n0 = nt * BN + static_cast<int>(cta_rank) * C::SUB_COLS * (CG - 1);   // + h * MMA_N per sub-MMA
         for (int kb = s.kb0; kb < s.kb1; ++kb) {
           if (!wait_bar(empty0 + stage * 8, phase ^ 1u, ctrl, p)) { ok = false; break; }
           const uint32_t a_dst = ring_addr + stage * C::STAGE_BYTES;
@@ -311,24 +337,34 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             const uint32_t bar = full0 + stage * 8;
             ptx::mbar_arrive_expect_tx(bar, C::STAGE_BYTES);
             if (!(p.test_starve && issued == 0)) ptx::tma_load_3d(a_dst, &tmA, bar, k0, m0, b);
-            if constexpr (B_KMAJOR) {
-              ptx::tma_load_3d(b_dst, &tmB, bar, k0, n0, b);
-            } else {
 #pragma unroll
-              for (int j = 0; j < C::BN_CTA / 64; ++j)
-                ptx::tma_load_3d(b_dst + j * (64 * BK * 2), &tmB, bar, n0 + j * 64, k0, b);
+            for (int h = 0; h < C::NSUB; ++h) {
+              const int nh = n0 + h * C::MMA_N;
+              const uint32_t dst = b_dst + h * C::SUB_B_BYTES;
+              if constexpr (B_KMAJOR) {
+                ptx::tma_load_3d(dst, &tmB, bar, k0, nh, b);
+              } else {
+#pragma unroll
+                for (int j = 0; j < C::SUB_COLS / 64; ++j)
+                  ptx::tma_load_3d(dst + j * (64 * BK * 2), &tmB, bar, nh + j * 64, k0, b);
+              }
             }
           } else {
             // both CTAs' bytes are counted on the leader's barrier
             if (cta_rank == 0) ptx::mbar_arrive_expect_tx(full0 + stage * 8, 2 * C::STAGE_BYTES);
             const uint32_t bar = full0_leader + stage * 8;
             if (!(p.test_starve && issued == 0)) ptx::tma_load_3d_pair(a_dst, &tmA, bar, k0, m0, b);
-            if constexpr (B_KMAJOR) {
-              ptx::tma_load_3d_pair(b_dst, &tmB, bar, k0, n0, b);
-            } else {
 #pragma unroll
-              for (int j = 0; j < C::BN_CTA / 64; ++j)
-                ptx::tma_load_3d_pair(b_dst + j * (64 * BK * 2), &tmB, bar, n0 + j * 64, k0, b);
+            for (int h = 0; h < C::NSUB; ++h) {
+              const int nh = n0 + h * C::MMA_N;
+              const uint32_t dst = b_dst + h * C::SUB_B_BYTES;
+              if constexpr (B_KMAJOR) {
+                ptx::tma_load_3d_pair(dst, &tmB, bar, k0, nh, b);
+              } else {
+#pragma unroll
+                for (int j = 0; j < C::SUB_COLS / 64; ++j)
+                  ptx::tma_load_3d_pair(dst + j * (64 * BK * 2), &tmB, bar, nh + j * 64, k0, b);
+              }
             }
           }
           ++issued;
@@ -374,6 +410,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       const uint32_t desc_hi = static_cast<uint32_t>(a_desc0 >> 32);      // same for A and B
       const uint32_t a_lo0 = static_cast<uint32_t>(a_desc0), b_lo0 = static_cast<uint32_t>(b_desc0);
       constexpr uint32_t STAGE_STEP = C::STAGE_BYTES >> 4;
+      constexpr uint32_t SUB_STEP = C::SUB_B_BYTES >> 4;                  // next sub-MMA's B columns
       constexpr uint32_t A_KSTEP = (UMMA_K * 2) >> 4;                     // +32 B inside the swizzle row
       constexpr uint32_t B_KSTEP = B_KMAJOR ? ((UMMA_K * 2) >> 4) : ((UMMA_K * 128) >> 4);   // or +16 k-rows
       const uint32_t full0 = ptx::smem_u32(&ctrl->full[0]);
@@ -394,14 +431,18 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           const uint32_t a_lo = a_lo0 + stage * STAGE_STEP;
           const uint32_t b_lo = b_lo0 + stage * STAGE_STEP;
           if (kb != last_kb || tail_nk == BK / UMMA_K) {
-            ptx::mma_f16<CG>(d_tmem, desc(a_lo), desc(b_lo), C::IDESC, accumulate);
-            ptx::mma_f16<CG>(d_tmem, desc(a_lo + A_KSTEP), desc(b_lo + B_KSTEP), C::IDESC, 1u);
-            ptx::mma_f16<CG>(d_tmem, desc(a_lo + 2 * A_KSTEP), desc(b_lo + 2 * B_KSTEP), C::IDESC, 1u);
-            ptx::mma_f16<CG>(d_tmem, desc(a_lo + 3 * A_KSTEP), desc(b_lo + 3 * B_KSTEP), C::IDESC, 1u);
+#pragma unroll
+            for (int k = 0; k < BK / UMMA_K; ++k)
+#pragma unroll
+              for (int h = 0; h < C::NSUB; ++h)
+                ptx::mma_f16<CG>(d_tmem + h * C::MMA_N, desc(a_lo + k * A_KSTEP), desc(b_lo + k * B_KSTEP + h * SUB_STEP),
+                                 C::IDESC, k == 0 ? accumulate : 1u);
           } else {
             for (int k = 0; k < tail_nk; ++k)     // K tail: skip 16-wide steps that are all padding
-              ptx::mma_f16<CG>(d_tmem, desc(a_lo + k * A_KSTEP), desc(b_lo + k * B_KSTEP), C::IDESC,
-                               (k > 0) ? 1u : accumulate);
+#pragma unroll
+              for (int h = 0; h < C::NSUB; ++h)
+                ptx::mma_f16<CG>(d_tmem + h * C::MMA_N, desc(a_lo + k * A_KSTEP), desc(b_lo + k * B_KSTEP + h * SUB_STEP),
+                                 C::IDESC, (k > 0) ? 1u : accumulate);
           }
           accumulate = 1u;
           ptx::tc_commit<CG>(empty0 + stage * 8);
@@ -412,8 +453,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         const uint32_t full_local = ptx::smem_u32(&ctrl->acc_full[acc]);
         ptx::tc_commit<CG>(full_local);
         if constexpr (CG == 2) ptx::tc_commit<CG>(ptx::mapa(full_local, 1));
-        acc ^= 1;
-        if (acc == 0) acc_phase ^= 1u;
+        if (++acc == C::ACC_BUFS) { acc = 0; acc_phase ^= 1u; }
       }
       if (!ok || *reinterpret_cast<volatile int*>(&ctrl->abort)) {
         // abort path: wait (bounded) until the MMAs issued so far have retired
@@ -425,11 +465,14 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     }
     __syncwarp();
   } else {
-    // ================================================================ epilogue (warps 2..5)
+    // ================================================================ epilogue (warps 2 and up)
+    const int ew = warp - 2;                    // epilogue warp index
     const int q = warp & 3;                     // TMEM lane quarter this warp may access
+    const int col_group = ew >> 2;              // which share of the tile's columns (wide tiles have two)
     const int row_in_tile = q * 32 + lane;
-    float* bias_s = bias_all + q * EPI_COLS;
-    const uint32_t stage_base = epi_addr + q * (EPI_BUFS * EPI_BUF_BYTES);
+    float* bias_s = bias_all + ew * EPI_COLS;
+    const uint32_t stage_base = epi_addr + ew * (C::EPI_BUFS * EPI_BUF_BYTES);
+    constexpr int CHUNKS_PER_GROUP = BN / EPI_COLS / C::EPI_COL_GROUPS;
     int store_buf = 0;
     int acc = 0;
     uint32_t acc_phase = 0;
@@ -453,10 +496,13 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                                                : ptx::smem_u32(&ctrl->acc_empty[acc]);
       int n_chunks = (p.N - n_base + EPI_COLS - 1) / EPI_COLS;    // chunks with at least one valid column
       if (n_chunks > BN / EPI_COLS) n_chunks = BN / EPI_COLS;
+      const int c_lo = col_group * CHUNKS_PER_GROUP;               // this warp's chunk range [c_lo, c_hi)
+      int c_hi = c_lo + CHUNKS_PER_GROUP;
+      if (c_hi > n_chunks) c_hi = n_chunks;
 
       bool reduce = false;        // this warp must run the epilogue from workspace partials
       int first_unit = 0, last_unit = 0;
-      if (!whole_tile) {
+      if (C::EPI_COL_GROUPS == 1 && !whole_tile) {     // (the host never splits the wide tile)
         // ---- split tile: park the fp32 partial, draw a ticket
         const int slot = 2 * s.unit + (s.head ? 0 : 1);
         float4* part = reinterpret_cast<float4*>(p.partials) + (static_cast<size_t>(slot) * (BM * BN / 4)) +
@@ -495,7 +541,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       }
 
       if (whole_tile || reduce) {
-        for (int c = 0; c < n_chunks; ++c) {
+        for (int c = c_lo; c < c_hi; ++c) {
           const int n0 = n_base + c * EPI_COLS;
           int n_valid = p.N - n0;
           if (n_valid > EPI_COLS) n_valid = EPI_COLS;
@@ -520,7 +566,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             ptx::tmem_ld_wait();
 #pragma unroll
             for (int j = 0; j < 32; ++j) { accv[j] = __uint_as_float(v0[j]); accv[32 + j] = __uint_as_float(v1[j]); }
-            if (c == n_chunks - 1) {     // accumulator fully read: hand the buffer back to the MMA warp
+            if (c == c_hi - 1) {         // this warp's share is read: its hand-back of the buffer to the MMA warp
               ptx::tc_fence_before();
               __syncwarp();
               if (lane == 0) {
@@ -542,7 +588,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             }
           }
           // staging buffer free again?  (the store issued two chunks ago has read it)
-          if (lane == 0) ptx::bulk_wait_group_read<EPI_BUFS - 1>();
+          if (lane == 0) ptx::bulk_wait_group_read<C::EPI_BUFS - 1>();
           __syncwarp();
           bias_s[lane] = bv0;
           bias_s[lane + 32] = bv1;
@@ -574,9 +620,9 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             if (warp_rows_valid) ptx::tma_store_3d(&tmD, buf_addr, n0, m_base + q * 32, b);   // clips rows >= M, cols >= N
             ptx::bulk_commit_group();
           }
-          store_buf = (store_buf + 1 == EPI_BUFS) ? 0 : store_buf + 1;
+          store_buf = (store_buf + 1 == C::EPI_BUFS) ? 0 : store_buf + 1;
         }
-        if (whole_tile && n_chunks == 0) {   // cannot happen (n_base < N), kept for symmetry of the protocol
+        if (whole_tile && c_lo >= c_hi) {    // none of this warp's columns exist (ragged N): still hand the buffer back
           ptx::tc_fence_before();
           __syncwarp();
           if (lane == 0) {
@@ -584,8 +630,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           }
         }
       }
-      acc ^= 1;
-      if (acc == 0) acc_phase ^= 1u;
+      if (++acc == C::ACC_BUFS) { acc = 0; acc_phase ^= 1u; }
     }
     if (lane == 0) ptx::bulk_wait_group<0>();   // all of this warp's stores have completed
     __syncwarp();

@@ -44,10 +44,10 @@ def check(ctx, oracle, p, exact=False, **tuning):
 
 SHAPES = [  # (M, N, K, batch)
     (128, 64, 64, 1), (1, 8, 8, 1), (127, 72, 8, 1), (129, 136, 200, 1), (200, 264, 72, 3), (384, 512, 256, 1),
-    (77, 1000, 1032, 2),
+    (77, 1000, 1032, 2), (520, 1544, 136, 1),
 ]
 PLANS = [dict(tile_n=64, cta_group=1), dict(tile_n=128, cta_group=1), dict(tile_n=256, cta_group=1),
-         dict(tile_n=128, cta_group=2), dict(tile_n=256, cta_group=2), dict()]
+         dict(tile_n=128, cta_group=2), dict(tile_n=256, cta_group=2), dict(tile_n=512, cta_group=2), dict()]
 
 
 @pytest.mark.parametrize("colmajor", [False, True])
@@ -65,6 +65,7 @@ def test_short_rings_wrap_correctly(ctx, oracle, stages):
     p = W.make(256, 256, 1024, seed=stages, A=SI, B=SI)
     check(ctx, oracle, p, exact=True, tile_n=128, cta_group=1, stages=stages, max_ctas=2)
     check(ctx, oracle, p, exact=True, tile_n=128, cta_group=2, stages=stages, max_ctas=2)
+    check(ctx, oracle, p, exact=True, tile_n=512, cta_group=2, stages=stages, max_ctas=2)
 
 
 def test_persistent_loop_few_ctas_and_raster(ctx, oracle):
@@ -72,6 +73,7 @@ def test_persistent_loop_few_ctas_and_raster(ctx, oracle):
     for gm in (1, 3, 8):
         check(ctx, oracle, p, exact=True, tile_n=128, cta_group=1, max_ctas=5, group_m=gm)
         check(ctx, oracle, p, exact=True, tile_n=256, cta_group=2, max_ctas=6, group_m=gm)
+        check(ctx, oracle, p, exact=True, tile_n=512, cta_group=2, max_ctas=4, group_m=gm)
 
 
 # ------------------------------------------------------------------ split-K / stream-K
@@ -112,6 +114,7 @@ def test_epilogue_variants(ctx, oracle, act, bias, residual):
                bias=None if bias is None else ("normal", 1.0), R=("normal", 1.0) if residual else None)
     check(ctx, oracle, p)
     check(ctx, oracle, p, tile_n=256, cta_group=2)
+    check(ctx, oracle, p, tile_n=512, cta_group=2)
 
 
 def test_activation_tails(ctx, oracle):
@@ -136,7 +139,7 @@ def test_beta_zero_ignores_R_and_alpha_zero_keeps_bias(ctx, oracle):
 def test_in_place_residual(ctx, oracle):
     p = W.make(260, 200, 128, batch=2, seed=4, alpha=0.5, beta=1.0, A=("uniform", 1.0), B=("uniform", 1.0), R=("normal", 1.0))
     r64, _ = PU.oracle_full(oracle, p)
-    for tuning in (dict(tile_n=64, cta_group=1), dict(tile_n=128, cta_group=2)):
+    for tuning in (dict(tile_n=64, cta_group=1), dict(tile_n=128, cta_group=2), dict(tile_n=512, cta_group=2)):
         dev = PU.to_device(p)
         dev["D"] = dev["R"]                           # D aliases R exactly
         ctx.set_tuning(reset=True)
