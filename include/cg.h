@@ -102,7 +102,9 @@ typedef struct cg_tuning {
   int cta_group; /* 1 = one CTA per 128-row tile, 2 = CTA pair sharing a 256-row tile       */
   int num_units; /* number of contiguous k-block ranges the iteration space is cut into:
                     = number of tiles -> data-parallel, a multiple of it -> split-K,
-                    anything else -> stream-K (cta_group 1 only)                            */
+                    anything else -> stream-K (tile_n <= 256)                               */
+  int dp_units;  /* with num_units: the first dp_units units are whole tiles, the other
+                    num_units - dp_units divide the remaining tiles' iterations evenly      */
   int stages;    /* depth of the shared-memory operand ring (clamped to what fits)          */
   int group_m;   /* raster: m-tiles walked before stepping to the next n-tile               */
   int max_ctas;  /* cap on the persistent grid (0 = one CTA per SM)                         */
@@ -115,6 +117,7 @@ typedef struct cg_plan_info {
   int grid;        /* CTAs launched                          */
   int num_tiles;   /* output tiles                           */
   int num_units;   /* k-block ranges (see cg_tuning)         */
+  int dp_units;    /* leading units that are whole tiles     */
   int k_blocks;    /* 64-wide k-blocks per tile              */
   int smem_bytes;  /* dynamic shared memory per CTA          */
   int launches;    /* kernels launched by the call (always 1)*/

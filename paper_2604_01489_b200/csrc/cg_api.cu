@@ -27,7 +27,7 @@ constexpr size_t DEFAULT_WORKSPACE = 64ull << 20;
 constexpr int MAX_TICKET_TILES = 1 << 16;          // tiles that may be split (4 tickets each)
 
 struct Plan {
-  int bn, cg, stages, group_m, num_units, grid, num_workers;
+  int bn, cg, stages, group_m, num_units, dp_units, grid, num_workers;
   int tiles_m, tiles_n, num_tiles, k_blocks, smem;
   bool b_kmajor;
 };
@@ -143,7 +143,9 @@ int make_map(cg_context* h, CUtensorMap* map, const void* base, uint64_t inner, 
 
 // ---- plan --------------------------------------------------------------------------
 
-size_t partial_need(int num_units, int bn) { return static_cast<size_t>(2) * num_units * BM * bn * sizeof(float); }
+size_t partial_need(long long split_units, int bn, int cgn) {
+  return static_cast<size_t>(2) * split_units * cgn * BM * bn * sizeof(float);
+}
 
 int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, Plan* pl) {
   const cg_tuning_t& t = h->tuning;
@@ -190,30 +192,49 @@ int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, Plan
   if (nt * k_blocks >= (1ll << 31) || nt >= (1ll << 29))
     return fail(h, CG_ERR_UNSUPPORTED, "problem too large: %lld tiles x %d k-blocks", nt, k_blocks);
   pl->num_tiles = static_cast<int>(nt);
-  const long long iters = nt * k_blocks;
 
   int max_workers = sms / cgn;
   if (max_workers < 1) max_workers = 1;
 
-  // units: data-parallel unless forced, or unless the tiles cannot fill the machine
-  long long units = pl->num_tiles;
+  // Units.  Default: whole tiles (data-parallel).  The tiles of a partial last wave are instead cut
+  // along K and spread over all workers; with fewer tiles than workers the whole problem is.
+  // Every such tile is cut into the same number of parts: parts of different tiles then walk the
+  // same k ranges at the same time and keep sharing A rows / B columns in L2 (ranges that are merely
+  // balanced do not, and the split phase becomes DRAM-bound).  Splitting needs k-blocks to spare,
+  // a tile count the ticket array covers and partial-tile space in the workspace.
+  const bool can_split = bn <= 256 && static_cast<long long>(pl->num_tiles) * cgn <= MAX_TICKET_TILES;
+  long long units = pl->num_tiles, dp = pl->num_tiles;
   if (t.num_units > 0) {
     units = t.num_units;
-  } else if (cgn == 1 && pl->num_tiles < max_workers && k_blocks >= 8 && pl->num_tiles <= MAX_TICKET_TILES) {
-    // stream-K: one contiguous range per SM, at least 4 k-blocks each
-    long long u = max_workers;
-    if (u > iters / 4) u = iters / 4;
-    if (u > pl->num_tiles && partial_need(static_cast<int>(u), bn) <= h->partial_bytes) units = u;
+    dp = t.dp_units;
+    if (dp > pl->num_tiles || dp > units) return fail(h, CG_ERR_INVALID_ARG, "dp_units exceeds the tile or unit count");
+    if (dp == pl->num_tiles && units != dp) return fail(h, CG_ERR_INVALID_ARG, "no iterations left for the split units");
+  } else if (can_split && k_blocks >= 8) {
+    const long long full = (pl->num_tiles / max_workers) * max_workers;       // tiles in full waves
+    const long long rem = pl->num_tiles - full;
+    if (rem > 0) {
+      long long parts = max_workers / rem;
+      if (parts > k_blocks / 4) parts = k_blocks / 4;                          // at least 4 k-blocks per part
+      if (parts >= 2 && partial_need(rem * parts, bn, cgn) <= h->partial_bytes) {
+        dp = full;
+        units = full + rem * parts;
+      }
+    }
   }
-  if (units > iters) units = iters;
-  if (units < 1) units = 1;
-  if (units != pl->num_tiles) {
-    if (cgn != 1) return fail(h, CG_ERR_UNSUPPORTED, "split plans need cta_group 1");
-    if (pl->num_tiles > MAX_TICKET_TILES || partial_need(static_cast<int>(units), bn) > h->partial_bytes)
+  if (dp > units) dp = units;
+  long long split_units = units - dp;
+  const long long rest = (pl->num_tiles - dp) * static_cast<long long>(k_blocks);   // iterations left for them
+  if (split_units > rest) split_units = rest;
+  if (split_units < 1 && rest > 0) split_units = 1;
+  units = dp + split_units;
+  if (split_units > 0 && split_units != pl->num_tiles - dp) {     // some unit boundary falls inside a tile
+    if (!can_split) return fail(h, CG_ERR_UNSUPPORTED, "this tile shape or tile count cannot be split along K");
+    if (partial_need(split_units, bn, cgn) > h->partial_bytes)
       return fail(h, CG_ERR_WORKSPACE, "split plan needs %zu bytes of workspace, handle has %zu",
-                  partial_need(static_cast<int>(units), bn), h->partial_bytes);
+                  partial_need(split_units, bn, cgn), h->partial_bytes);
   }
   pl->num_units = static_cast<int>(units);
+  pl->dp_units = static_cast<int>(dp);
   pl->num_workers = pl->num_units < max_workers ? pl->num_units : max_workers;
   pl->grid = pl->num_workers * cgn;
 
@@ -276,9 +297,11 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   p.k_blocks = pl.k_blocks;
   p.group_m = pl.group_m;
   p.num_units = pl.num_units;
-  const long long iters = static_cast<long long>(pl.num_tiles) * pl.k_blocks;
-  p.unit_q = static_cast<int>(iters / pl.num_units);
-  p.unit_r = static_cast<int>(iters % pl.num_units);
+  p.dp_units = pl.dp_units;
+  const long long rest = static_cast<long long>(pl.num_tiles - pl.dp_units) * pl.k_blocks;
+  const int split_units = pl.num_units - pl.dp_units;
+  p.unit_q = split_units > 0 ? static_cast<int>(rest / split_units) : 1;
+  p.unit_r = split_units > 0 ? static_cast<int>(rest % split_units) : 0;
   p.num_workers = pl.num_workers;
   p.stages = pl.stages;
   p.alpha = alpha; p.beta = beta;
@@ -310,7 +333,8 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
 
   cg_plan_info_t& lp = h->last_plan;
   lp.tile_m = BM * pl.cg; lp.tile_n = pl.bn; lp.cta_group = pl.cg; lp.stages = pl.stages; lp.group_m = pl.group_m;
-  lp.grid = pl.grid; lp.num_tiles = pl.num_tiles; lp.num_units = pl.num_units; lp.k_blocks = pl.k_blocks;
+  lp.grid = pl.grid; lp.num_tiles = pl.num_tiles; lp.num_units = pl.num_units; lp.dp_units = pl.dp_units;
+  lp.k_blocks = pl.k_blocks;
   lp.smem_bytes = pl.smem; lp.launches = 1;
   h->last_status = CG_OK;
   h->last_msg[0] = 0;
@@ -426,7 +450,7 @@ int cg_set_tuning(cg_handle_t h, const cg_tuning_t* t) {
     return CG_OK;
   }
   if ((t->tile_n != 0 && t->tile_n != 64 && t->tile_n != 128 && t->tile_n != 256 && t->tile_n != 512) || t->cta_group < 0 ||
-      t->cta_group > 2 || t->num_units < 0 || t->stages < 0 || t->group_m < 0 || t->max_ctas < 0)
+      t->cta_group > 2 || t->num_units < 0 || t->dp_units < 0 || t->stages < 0 || t->group_m < 0 || t->max_ctas < 0)
     return fail(h, CG_ERR_INVALID_ARG, "bad tuning values");
   h->tuning = *t;
   return CG_OK;

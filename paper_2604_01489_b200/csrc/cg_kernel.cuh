@@ -15,9 +15,11 @@
 //                      lanes) of its quarter and never synchronises with the other warps.
 //
 // Work decomposition: the iteration space (tile, k-block) is linearised tile-major and cut
-// into `num_units` contiguous, balanced ranges; worker w takes units w, w + W, ...  A unit
-// that covers whole tiles is plain data-parallel work; a unit boundary inside a tile makes
-// that tile split-K / stream-K: every contributor writes its fp32 partial to the workspace,
+// into `num_units` contiguous ranges: the first `dp_units` are whole tiles (the full waves of a
+// data-parallel schedule), the rest divide the remaining iterations evenly (the partial last
+// wave, spread over all workers); worker w takes units w, w + W, ...  A unit that covers whole
+// tiles is plain data-parallel work; a unit boundary inside a tile makes that tile
+// split-K / stream-K: every contributor writes its fp32 partial to the workspace,
 // draws a ticket, and the last one to arrive sums all partials in unit order (deterministic)
 // and runs the epilogue.  Nobody ever waits for another CTA.
 //
@@ -61,7 +63,8 @@ struct KernelParams {
   int k_blocks;           // ceil(K / 64)
   int group_m;            // raster: m-tiles walked before the next n-tile
   int num_units;          // contiguous k-block ranges
-  int unit_q, unit_r;     // start(u) = u*unit_q + min(u, unit_r)
+  int dp_units;           // the first dp_units units are whole tiles (unit u = tile u) ...
+  int unit_q, unit_r;     // ... the rest cut the remaining iterations evenly: start = base + v*q + min(v, r)
   int num_workers;        // CTAs (CG == 1) or CTA pairs (CG == 2)
   int stages;
   float alpha, beta;
@@ -69,8 +72,8 @@ struct KernelParams {
   int bias_bf16;
   const void* bias;
   const __nv_bfloat16* R;
-  float* partials;        // [2 * num_units][BM * BN] fp32 partial tiles
-  int* tickets;           // [num_tiles * 4], zero between launches
+  float* partials;        // [2 * (num_units - dp_units)][CG][BM * BN] fp32 partial tiles
+  int* tickets;           // [num_tiles * CG * 4], zero between launches
   int* status;
   long long wait_limit;   // clock cycles before a wait gives up
   int test_starve;        // test hook: the producer withholds the first A load, so `full[0]` never completes
@@ -122,11 +125,16 @@ static_assert(sizeof(Ctrl) <= CTRL_BYTES, "control block");
 // ---------------------------------------------------------------- scheduling helpers
 
 __device__ __forceinline__ int unit_start(const KernelParams& p, int u) {
-  return u * p.unit_q + (u < p.unit_r ? u : p.unit_r);
+  if (u <= p.dp_units) return u * p.k_blocks;
+  const int v = u - p.dp_units;
+  return p.dp_units * p.k_blocks + v * p.unit_q + (v < p.unit_r ? v : p.unit_r);
 }
 __device__ __forceinline__ int unit_of_iter(const KernelParams& p, int it) {
+  const int base = p.dp_units * p.k_blocks;
+  if (it < base) return it / p.k_blocks;
+  const int rel = it - base;
   const int big = p.unit_r * (p.unit_q + 1);
-  return it < big ? it / (p.unit_q + 1) : p.unit_r + (it - big) / p.unit_q;
+  return p.dp_units + (rel < big ? rel / (p.unit_q + 1) : p.unit_r + (rel - big) / p.unit_q);
 }
 
 struct Segment {
@@ -504,9 +512,10 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       int first_unit = 0, last_unit = 0;
       if (C::EPI_COL_GROUPS == 1 && !whole_tile) {     // (the host never splits the wide tile)
         // ---- split tile: park the fp32 partial, draw a ticket
-        const int slot = 2 * s.unit + (s.head ? 0 : 1);
+        const int slot = (2 * (s.unit - p.dp_units) + (s.head ? 0 : 1)) * CG + static_cast<int>(cta_rank);
         float4* part = reinterpret_cast<float4*>(p.partials) + (static_cast<size_t>(slot) * (BM * BN / 4)) +
                        static_cast<size_t>(q) * (32 * BN / 4);
+        int* ticket = p.tickets + (s.tile * CG + static_cast<int>(cta_rank)) * 4 + q;
         for (int c = 0; c < BN / 32; ++c) {
           uint32_t v[32];
           ptx::tmem_ld_32x32b_x32(taddr + c * 32, v);
@@ -526,11 +535,11 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           first_unit = unit_of_iter(p, s.tile * p.k_blocks);
           last_unit = unit_of_iter(p, (s.tile + 1) * p.k_blocks - 1);
           const int parts = last_unit - first_unit + 1;
-          const int old = atomicAdd(p.tickets + s.tile * 4 + q, 1);
+          const int old = atomicAdd(ticket, 1);
           last = (old == parts - 1) ? 1 : 0;
           if (last) {
             __threadfence();
-            atomicExch(p.tickets + s.tile * 4 + q, 0);     // self-reset for the next launch
+            atomicExch(ticket, 0);     // self-reset for the next launch
           }
         }
         last = __shfl_sync(0xFFFFFFFFu, last, 0);
@@ -577,7 +586,8 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 #pragma unroll
             for (int j = 0; j < EPI_COLS; ++j) accv[j] = 0.0f;
             for (int u = first_unit; u <= last_unit; ++u) {     // fixed order => deterministic sum
-              const int slot = 2 * u + (unit_start(p, u) >= s.tile * p.k_blocks ? 0 : 1);
+              const int slot = (2 * (u - p.dp_units) + (unit_start(p, u) >= s.tile * p.k_blocks ? 0 : 1)) * CG +
+                               static_cast<int>(cta_rank);
               const float4* part = reinterpret_cast<const float4*>(p.partials) +
                                    (static_cast<size_t>(slot) * (BM * BN / 4)) + static_cast<size_t>(q) * (32 * BN / 4);
 #pragma unroll

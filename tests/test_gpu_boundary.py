@@ -74,8 +74,11 @@ def test_tuning_validation_and_plan_report(cg, ctx):
     ctx.set_tuning(tile_n=512, cta_group=1)                              # the wide tile is for CTA pairs only
     assert cg.cg_gemm_epilogue(ctx.handle, dev["A"], dev["B"], None, None, dev["D"], 256, 256, 256, 1, 1.0, 0.0, 0) == cg.CG_ERR_INVALID_ARG
     ctx.set_tuning(reset=True)
-    ctx.set_tuning(tile_n=128, cta_group=2, num_units=3)                 # split plans are 1-CTA only
+    ctx.set_tuning(tile_n=512, cta_group=2, num_units=3)                 # the wide tile cannot be split along K
     assert cg.cg_gemm_epilogue(ctx.handle, dev["A"], dev["B"], None, None, dev["D"], 256, 256, 256, 1, 1.0, 0.0, 0) == cg.CG_ERR_UNSUPPORTED
+    ctx.set_tuning(reset=True)
+    ctx.set_tuning(tile_n=128, cta_group=1, num_units=6, dp_units=5)     # more whole-tile units than tiles
+    assert cg.cg_gemm_epilogue(ctx.handle, dev["A"], dev["B"], None, None, dev["D"], 256, 256, 256, 1, 1.0, 0.0, 0) == cg.CG_ERR_INVALID_ARG
     ctx.set_tuning(reset=True)
     ctx.set_tuning(tile_n=128, cta_group=1, num_units=6, stages=3, group_m=2)
     PU.run_gpu(ctx, p, dev)

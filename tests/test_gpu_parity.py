@@ -85,6 +85,35 @@ def test_split_and_stream_k(ctx, oracle, units):
     assert plan["num_units"] == units and plan["num_tiles"] == 4
 
 
+@pytest.mark.parametrize("units", [2, 3, 5, 8, 11])
+def test_split_and_stream_k_on_cta_pairs(ctx, oracle, units):
+    p = W.make(512, 512, 640, seed=units, act=W.ACT_RELU, alpha=2.0, beta=-1.0, A=SI, B=SI, bias=SI, R=SI)
+    plan = check(ctx, oracle, p, exact=True, tile_n=256, cta_group=2, num_units=units)     # 4 pair tiles x 10 k-blocks
+    assert plan["num_units"] == units and plan["num_tiles"] == 4 and plan["cta_group"] == 2
+    check(ctx, oracle, p, exact=True, tile_n=128, cta_group=2, num_units=units + 8, max_ctas=6)
+
+
+@pytest.mark.parametrize("cta_group,dp,units", [(1, 4, 7), (1, 6, 9), (1, 7, 8), (2, 2, 5), (2, 3, 7), (1, 8, 8), (1, 0, 8)])
+def test_hybrid_whole_tiles_then_stream_k(ctx, oracle, cta_group, dp, units):
+    """The first `dp` units are whole tiles, the remaining tiles are cut along K."""
+    M = 512 if cta_group == 1 else 1024
+    p = W.make(M, 256, 1032, seed=dp * 10 + units, act=W.FLAG_B_COLMAJOR | W.ACT_RELU, A=SI, B=SI, bias=SI)   # 8 or 4 tiles
+    tiles = 8 if cta_group == 1 else 4
+    plan = check(ctx, oracle, p, exact=True, tile_n=128 if cta_group == 1 else 256, cta_group=cta_group, num_units=units,
+                 dp_units=dp, max_ctas=3 * cta_group)
+    assert plan["num_tiles"] == tiles and plan["dp_units"] == dp and plan["num_units"] == units
+
+
+def test_heuristic_splits_a_thin_last_wave(ctx, oracle):
+    """14 pair tiles on 4 CTA pairs = 3.5 waves: three data-parallel waves, the last two tiles stream-K."""
+    p = W.make(1792, 512, 1024, seed=77, act=W.ACT_SILU, A=("normal", 1.0), B=("normal", 0.05), bias=("normal", 1.0))
+    plan = check(ctx, oracle, p, tile_n=256, cta_group=2, max_ctas=8)
+    assert plan["num_tiles"] == 14 and plan["dp_units"] == 12 and plan["num_units"] == 16
+    p2 = W.make(1536, 512, 1024, seed=78, A=SI, B=SI)                       # 12 tiles = exactly 3 waves: no split
+    plan = check(ctx, oracle, p2, exact=True, tile_n=256, cta_group=2, max_ctas=8)
+    assert plan["dp_units"] == 12 and plan["num_units"] == 12
+
+
 def test_stream_k_with_fewer_ctas_than_units_and_colmajor(ctx, oracle):
     p = W.make(200, 320, 1032, batch=2, seed=3, act=W.FLAG_B_COLMAJOR, A=SI, B=SI, alpha=1.0, beta=2.0, R=SI)
     check(ctx, oracle, p, exact=True, tile_n=64, cta_group=1, num_units=37, max_ctas=4)
