@@ -229,8 +229,8 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 //   t = alpha*acc + bias[n];  u = act(t);  v = u + beta*R[m,n]
 template <int ACT, bool HAS_R>
 __device__ __forceinline__ void epilogue_chunk(const float (&acc)[EPI_COLS], const float* bias_s, float alpha,
-                                               float beta, const __nv_bfloat16* r_row, int n_valid,
-                                               bool row_valid, uint32_t stage_row_addr, int lane) {
+                                               float beta, const uint4 (&rq)[EPI_COLS / 8], uint32_t stage_row_addr,
+                                               int lane) {
 #pragma unroll
   for (int c = 0; c < EPI_COLS / 8; ++c) {       // 8 columns = one 16-byte chunk of bf16
     float v[8];
@@ -239,15 +239,12 @@ __device__ __forceinline__ void epilogue_chunk(const float (&acc)[EPI_COLS], con
     const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
 #pragma unroll
     for (int j = 0; j < 8; ++j) v[j] = activate<ACT>(fmaf(alpha, acc[c * 8 + j], bb[j]));
-    if constexpr (HAS_R) {
-      if (row_valid && c * 8 < n_valid) {
-        const uint4 rr = *reinterpret_cast<const uint4*>(r_row + c * 8);
-        const uint32_t w[4] = {rr.x, rr.y, rr.z, rr.w};
+    if constexpr (HAS_R) {      // residual: eight bf16 of this row, fetched before the accumulator was read
+      const uint32_t w[4] = {rq[c].x, rq[c].y, rq[c].z, rq[c].w};
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          v[2 * j] = fmaf(beta, __uint_as_float(w[j] << 16), v[2 * j]);
-          v[2 * j + 1] = fmaf(beta, __uint_as_float(w[j] & 0xFFFF0000u), v[2 * j + 1]);
-        }
+      for (int j = 0; j < 4; ++j) {
+        v[2 * j] = fmaf(beta, __uint_as_float(w[j] << 16), v[2 * j]);
+        v[2 * j + 1] = fmaf(beta, __uint_as_float(w[j] & 0xFFFF0000u), v[2 * j + 1]);
       }
     }
     const uint32_t o0 = pack_bf16x2(v[0], v[1]), o1 = pack_bf16x2(v[2], v[3]);
@@ -488,7 +485,30 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     Segment s;
     bool ok = true;
     const bool has_r = (p.beta != 0.0f);
+    // Pulls this thread's row of a tile's residual (its share of the columns) into L2.
+    auto prefetch_residual = [&](const Segment& sg) {
+      int pb, pmt, pnt;
+      decode_tile(p, sg.tile, pb, pmt, pnt);
+      const int pm = pmt * (BM * CG) + static_cast<int>(cta_rank) * BM + row_in_tile;
+      if (pm >= p.M) return;
+      const int col0 = pnt * BN + col_group * (CHUNKS_PER_GROUP * EPI_COLS);
+      const char* row = reinterpret_cast<const char*>(p.R + (static_cast<size_t>(pb) * p.M + pm) * p.N);
+#pragma unroll
+      for (int j = 0; j < CHUNKS_PER_GROUP; ++j)                       // one 128-byte line per 64 columns
+        if (col0 + j * EPI_COLS < p.N)
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(row + static_cast<size_t>(col0 + j * EPI_COLS) * 2));
+    };
+    if (has_r) {                 // first tile: nothing ran ahead of it
+      WorkIter peek = wi;
+      Segment s0;
+      if (peek.next(s0)) prefetch_residual(s0);
+    }
     while (ok && wi.next(s)) {
+      if (has_r) {               // the tile after this one: a whole main loop ahead of its use
+        WorkIter peek = wi;
+        Segment s1;
+        if (peek.next(s1)) prefetch_residual(s1);
+      }
       int b, mt, nt;
       decode_tile(p, s.tile, b, mt, nt);
       const int m_base = mt * (BM * CG) + static_cast<int>(cta_rank) * BM;   // first row of this CTA's slab
@@ -567,6 +587,15 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
               if (lane + 32 < n_valid) bv1 = __ldg(bp + n0 + lane + 32);
             }
           }
+          // residual for this chunk: issued now so that its latency overlaps the accumulator read
+          uint4 rq[EPI_COLS / 8];
+          if (has_r) {
+            const uint4* r_row = reinterpret_cast<const uint4*>(
+                p.R + (static_cast<size_t>(b) * p.M + (row_valid ? m : 0)) * p.N + n0);
+#pragma unroll
+            for (int j = 0; j < EPI_COLS / 8; ++j)
+              rq[j] = (row_valid && j * 8 < n_valid) ? r_row[j] : make_uint4(0u, 0u, 0u, 0u);
+          }
           float accv[EPI_COLS];
           if (whole_tile) {
             uint32_t v0[32], v1[32];
@@ -605,23 +634,22 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           __syncwarp();
           const uint32_t buf_addr = stage_base + store_buf * EPI_BUF_BYTES;
           const uint32_t row_addr = buf_addr + lane * 128;
-          const __nv_bfloat16* r_row = has_r ? p.R + (static_cast<size_t>(b) * p.M + (row_valid ? m : 0)) * p.N + n0 : nullptr;
           switch (p.act) {
             case ACT_RELU:
-              if (has_r) epilogue_chunk<ACT_RELU, true>(accv, bias_s, p.alpha, p.beta, r_row, n_valid, row_valid, row_addr, lane);
-              else epilogue_chunk<ACT_RELU, false>(accv, bias_s, p.alpha, p.beta, r_row, n_valid, row_valid, row_addr, lane);
+              if (has_r) epilogue_chunk<ACT_RELU, true>(accv, bias_s, p.alpha, p.beta, rq, row_addr, lane);
+              else epilogue_chunk<ACT_RELU, false>(accv, bias_s, p.alpha, p.beta, rq, row_addr, lane);
               break;
             case ACT_GELU_TANH:
-              if (has_r) epilogue_chunk<ACT_GELU_TANH, true>(accv, bias_s, p.alpha, p.beta, r_row, n_valid, row_valid, row_addr, lane);
-              else epilogue_chunk<ACT_GELU_TANH, false>(accv, bias_s, p.alpha, p.beta, r_row, n_valid, row_valid, row_addr, lane);
+              if (has_r) epilogue_chunk<ACT_GELU_TANH, true>(accv, bias_s, p.alpha, p.beta, rq, row_addr, lane);
+              else epilogue_chunk<ACT_GELU_TANH, false>(accv, bias_s, p.alpha, p.beta, rq, row_addr, lane);
               break;
             case ACT_SILU:
-              if (has_r) epilogue_chunk<ACT_SILU, true>(accv, bias_s, p.alpha, p.beta, r_row, n_valid, row_valid, row_addr, lane);
-              else epilogue_chunk<ACT_SILU, false>(accv, bias_s, p.alpha, p.beta, r_row, n_valid, row_valid, row_addr, lane);
+              if (has_r) epilogue_chunk<ACT_SILU, true>(accv, bias_s, p.alpha, p.beta, rq, row_addr, lane);
+              else epilogue_chunk<ACT_SILU, false>(accv, bias_s, p.alpha, p.beta, rq, row_addr, lane);
               break;
             default:
-              if (has_r) epilogue_chunk<ACT_NONE, true>(accv, bias_s, p.alpha, p.beta, r_row, n_valid, row_valid, row_addr, lane);
-              else epilogue_chunk<ACT_NONE, false>(accv, bias_s, p.alpha, p.beta, r_row, n_valid, row_valid, row_addr, lane);
+              if (has_r) epilogue_chunk<ACT_NONE, true>(accv, bias_s, p.alpha, p.beta, rq, row_addr, lane);
+              else epilogue_chunk<ACT_NONE, false>(accv, bias_s, p.alpha, p.beta, rq, row_addr, lane);
               break;
           }
           ptx::fence_proxy_async_smem();      // my generic-proxy writes -> visible to the TMA store
