@@ -24,7 +24,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 constexpr size_t DEFAULT_WORKSPACE = 64ull << 20;
-constexpr int MAX_TICKET_TILES = 1 << 16;          // tiles that may be split (4 tickets each)
+constexpr int MAX_TICKET_TILES = 1 << 16;          // (tile, CTA) pairs that may be split
+constexpr int TICKETS_PER_TILE = 8;                // one ticket per epilogue warp slot
 
 struct Plan {
   int bn, cg, stages, group_m, num_units, dp_units, grid, num_workers;
@@ -381,7 +382,7 @@ int cg_create(cg_handle_t* out, int device, size_t workspace_bytes) {
   h->encode = reinterpret_cast<EncodeTiledFn>(fn);
 
   if (workspace_bytes == 0) workspace_bytes = DEFAULT_WORKSPACE;
-  const size_t ticket_bytes = static_cast<size_t>(MAX_TICKET_TILES) * 4 * sizeof(int);
+  const size_t ticket_bytes = static_cast<size_t>(MAX_TICKET_TILES) * TICKETS_PER_TILE * sizeof(int);
   if (workspace_bytes < ticket_bytes + (1u << 20)) workspace_bytes = ticket_bytes + (1u << 20);
   h->workspace_bytes = workspace_bytes;
   if (cudaMalloc(reinterpret_cast<void**>(&h->workspace), workspace_bytes) != cudaSuccess ||
@@ -477,7 +478,7 @@ int cg_last_error(cg_handle_t h, int sync, char* buf, size_t len) {
     } else if (dev != 0) {
       code = fail(h, dev, "a bounded wait inside the kernel expired (device status %d)", dev);
       // a timed-out split tile may have left tickets behind
-      cudaMemset(h->tickets, 0, static_cast<size_t>(MAX_TICKET_TILES) * 4 * sizeof(int));
+      cudaMemset(h->tickets, 0, static_cast<size_t>(MAX_TICKET_TILES) * TICKETS_PER_TILE * sizeof(int));
     } else {
       code = CG_OK;
       if (h->last_status == CG_OK) h->last_msg[0] = 0;
@@ -518,7 +519,7 @@ namespace {
 constexpr int NOALLOC_TILE_N = 128;
 constexpr int NOALLOC_MAX_TILES = 4096;                                  // tiles that may be split
 constexpr size_t NOALLOC_STATUS_BYTES = 256;
-constexpr size_t NOALLOC_TICKET_BYTES = static_cast<size_t>(NOALLOC_MAX_TILES) * 4 * sizeof(int);
+constexpr size_t NOALLOC_TICKET_BYTES = static_cast<size_t>(NOALLOC_MAX_TILES) * TICKETS_PER_TILE * sizeof(int);
 constexpr size_t NOALLOC_PARTIAL_BYTES = 8u << 20;                       // 8 MiB of fp32 partial tiles
 constexpr int NOALLOC_MAX_DEVICES = 64;
 
@@ -624,7 +625,7 @@ extern "C" int cg_gemm_epilogue_noalloc(const void* A, const void* B, const void
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (parts > 1) {
     // the array keeps whatever the previous call left: tickets must start at zero
-    const cudaError_t e = cudaMemsetAsync(h->tickets, 0, static_cast<size_t>(tiles) * 4 * sizeof(int), st);
+    const cudaError_t e = cudaMemsetAsync(h->tickets, 0, static_cast<size_t>(tiles) * TICKETS_PER_TILE * sizeof(int), st);
     if (e != cudaSuccess) { set_err(err, err_len, cudaGetErrorString(e)); return CG_ERR_CUDA; }
   }
   rc = launch(h, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, st);

@@ -73,7 +73,7 @@ struct KernelParams {
   const void* bias;
   const __nv_bfloat16* R;
   float* partials;        // [2 * (num_units - dp_units)][CG][BM * BN] fp32 partial tiles
-  int* tickets;           // [num_tiles * CG * 4], zero between launches
+  int* tickets;           // [num_tiles * CG * 8] (one per epilogue warp slot), zero between launches
   int* status;
   long long wait_limit;   // clock cycles before a wait gives up
   int test_starve;        // test hook: the producer withholds the first A load, so `full[0]` never completes
@@ -93,7 +93,9 @@ struct Cfg {
   static constexpr int B_BYTES = NSUB * SUB_B_BYTES;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int ACC_BUFS = (2 * BN <= 512) ? 2 : 1;   // accumulator buffers in TMEM
-  static constexpr int EPI_WARPS = (BN == 512) ? 8 : 4;
+  // Two warps per TMEM lane quarter (each takes half the tile's columns) once a tile has at least
+  // two 64-column chunks: one warp per scheduler cannot hide the TMEM / shared-memory / store latencies.
+  static constexpr int EPI_WARPS = (BN >= 128) ? 8 : 4;
   static constexpr int EPI_COL_GROUPS = EPI_WARPS / 4;       // warps per TMEM lane quarter
   static constexpr int EPI_BUFS = (EPI_WARPS == 4) ? 2 : 1;  // staging buffers per warp
   static constexpr int NUM_THREADS = 64 + 32 * EPI_WARPS;
@@ -517,6 +519,27 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       const bool row_valid = m < p.M;
       const bool warp_rows_valid = (m_base + q * 32) < p.M;
       const bool whole_tile = (s.kb0 == 0 && s.kb1 == p.k_blocks);
+      // bias of this warp's columns: two values per lane and chunk, fetched before the wait for the
+      // accumulator so that the loads are off the critical path
+      float bias_reg[2 * CHUNKS_PER_GROUP];
+#pragma unroll
+      for (int j = 0; j < CHUNKS_PER_GROUP; ++j) {
+        const int col = n_base + (col_group * CHUNKS_PER_GROUP + j) * EPI_COLS + lane;
+        float b0 = 0.0f, b1 = 0.0f;
+        if (p.bias != nullptr) {
+          if (p.bias_bf16) {
+            const __nv_bfloat16* bp = static_cast<const __nv_bfloat16*>(p.bias);
+            if (col < p.N) b0 = __bfloat162float(bp[col]);
+            if (col + 32 < p.N) b1 = __bfloat162float(bp[col + 32]);
+          } else {
+            const float* bp = static_cast<const float*>(p.bias);
+            if (col < p.N) b0 = __ldg(bp + col);
+            if (col + 32 < p.N) b1 = __ldg(bp + col + 32);
+          }
+        }
+        bias_reg[2 * j] = b0;
+        bias_reg[2 * j + 1] = b1;
+      }
       if (!wait_bar(ptx::smem_u32(&ctrl->acc_full[acc]), acc_phase, ctrl, p)) { ok = false; break; }
       ptx::tc_fence_after();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(acc * BN);
@@ -530,13 +553,14 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 
       bool reduce = false;        // this warp must run the epilogue from workspace partials
       int first_unit = 0, last_unit = 0;
-      if (C::EPI_COL_GROUPS == 1 && !whole_tile) {     // (the host never splits the wide tile)
+      if (!whole_tile) {
         // ---- split tile: park the fp32 partial, draw a ticket
         const int slot = (2 * (s.unit - p.dp_units) + (s.head ? 0 : 1)) * CG + static_cast<int>(cta_rank);
         float4* part = reinterpret_cast<float4*>(p.partials) + (static_cast<size_t>(slot) * (BM * BN / 4)) +
                        static_cast<size_t>(q) * (32 * BN / 4);
-        int* ticket = p.tickets + (s.tile * CG + static_cast<int>(cta_rank)) * 4 + q;
-        for (int c = 0; c < BN / 32; ++c) {
+        int* ticket = p.tickets + ((s.tile * CG + static_cast<int>(cta_rank)) * 4 + q) * 2 + col_group;
+        constexpr int GROUPS32 = BN / 32 / C::EPI_COL_GROUPS;      // 32-column groups in this warp's share
+        for (int c = col_group * GROUPS32; c < (col_group + 1) * GROUPS32; ++c) {
           uint32_t v[32];
           ptx::tmem_ld_32x32b_x32(taddr + c * 32, v);
           ptx::tmem_ld_wait();
@@ -574,19 +598,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           const int n0 = n_base + c * EPI_COLS;
           int n_valid = p.N - n0;
           if (n_valid > EPI_COLS) n_valid = EPI_COLS;
-          // bias for this chunk: two values per lane, staged per warp
-          float bv0 = 0.0f, bv1 = 0.0f;
-          if (p.bias != nullptr) {
-            if (p.bias_bf16) {
-              const __nv_bfloat16* bp = static_cast<const __nv_bfloat16*>(p.bias);
-              if (lane < n_valid) bv0 = __bfloat162float(bp[n0 + lane]);
-              if (lane + 32 < n_valid) bv1 = __bfloat162float(bp[n0 + lane + 32]);
-            } else {
-              const float* bp = static_cast<const float*>(p.bias);
-              if (lane < n_valid) bv0 = __ldg(bp + n0 + lane);
-              if (lane + 32 < n_valid) bv1 = __ldg(bp + n0 + lane + 32);
-            }
-          }
+          const float bv0 = bias_reg[2 * (c - c_lo)], bv1 = bias_reg[2 * (c - c_lo) + 1];   // fetched at tile start
           // residual for this chunk: issued now so that its latency overlaps the accumulator read
           uint4 rq[EPI_COLS / 8];
           if (has_r) {
