@@ -227,12 +227,11 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&h);
 }
 
-// One warp, one 64-column chunk: acc (thread = row, 64 fp32) -> bf16 in swizzled staging.
+// One warp, one 64-column chunk: acc (thread = row, 64 fp32) -> 64 bf16 packed in 32 registers.
 //   t = alpha*acc + bias[n];  u = act(t);  v = u + beta*R[m,n]
 template <int ACT, bool HAS_R>
 __device__ __forceinline__ void epilogue_chunk(const float (&acc)[EPI_COLS], const float* bias_s, float alpha,
-                                               float beta, const uint4 (&rq)[EPI_COLS / 8], uint32_t stage_row_addr,
-                                               int lane) {
+                                               float beta, const uint4 (&rq)[EPI_COLS / 8], uint32_t (&out)[EPI_COLS / 2]) {
 #pragma unroll
   for (int c = 0; c < EPI_COLS / 8; ++c) {       // 8 columns = one 16-byte chunk of bf16
     float v[8];
@@ -249,11 +248,19 @@ __device__ __forceinline__ void epilogue_chunk(const float (&acc)[EPI_COLS], con
         v[2 * j + 1] = fmaf(beta, __uint_as_float(w[j] & 0xFFFF0000u), v[2 * j + 1]);
       }
     }
-    const uint32_t o0 = pack_bf16x2(v[0], v[1]), o1 = pack_bf16x2(v[2], v[3]);
-    const uint32_t o2 = pack_bf16x2(v[4], v[5]), o3 = pack_bf16x2(v[6], v[7]);
-    // 128-byte swizzle: 16-byte chunk index XOR (row mod 8); staging rows are 128 B, row = lane
+#pragma unroll
+    for (int j = 0; j < 4; ++j) out[c * 4 + j] = pack_bf16x2(v[2 * j], v[2 * j + 1]);
+  }
+}
+
+// The packed chunk -> this thread's row of the staging buffer.  128-byte swizzle: 16-byte chunk
+// index XOR (row mod 8); staging rows are 128 B, row = lane (conflict-free, matches the D tensor map).
+__device__ __forceinline__ void stage_chunk(const uint32_t (&out)[EPI_COLS / 2], uint32_t stage_row_addr, int lane) {
+#pragma unroll
+  for (int c = 0; c < EPI_COLS / 8; ++c) {
     const uint32_t addr = stage_row_addr + (static_cast<uint32_t>(c ^ (lane & 7)) << 4);
-    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(out[c * 4]), "r"(out[c * 4 + 1]),
+                 "r"(out[c * 4 + 2]), "r"(out[c * 4 + 3]) : "memory");
   }
 }
 
@@ -638,32 +645,34 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
               }
             }
           }
-          // staging buffer free again?  (the store issued two chunks ago has read it)
-          if (lane == 0) ptx::bulk_wait_group_read<C::EPI_BUFS - 1>();
-          __syncwarp();
           bias_s[lane] = bv0;
           bias_s[lane + 32] = bv1;
           __syncwarp();
-          const uint32_t buf_addr = stage_base + store_buf * EPI_BUF_BYTES;
-          const uint32_t row_addr = buf_addr + lane * 128;
+          uint32_t outw[EPI_COLS / 2];
           switch (p.act) {
             case ACT_RELU:
-              if (has_r) epilogue_chunk<ACT_RELU, true>(accv, bias_s, p.alpha, p.beta, rq, row_addr, lane);
-              else epilogue_chunk<ACT_RELU, false>(accv, bias_s, p.alpha, p.beta, rq, row_addr, lane);
+              if (has_r) epilogue_chunk<ACT_RELU, true>(accv, bias_s, p.alpha, p.beta, rq, outw);
+              else epilogue_chunk<ACT_RELU, false>(accv, bias_s, p.alpha, p.beta, rq, outw);
               break;
             case ACT_GELU_TANH:
-              if (has_r) epilogue_chunk<ACT_GELU_TANH, true>(accv, bias_s, p.alpha, p.beta, rq, row_addr, lane);
-              else epilogue_chunk<ACT_GELU_TANH, false>(accv, bias_s, p.alpha, p.beta, rq, row_addr, lane);
+              if (has_r) epilogue_chunk<ACT_GELU_TANH, true>(accv, bias_s, p.alpha, p.beta, rq, outw);
+              else epilogue_chunk<ACT_GELU_TANH, false>(accv, bias_s, p.alpha, p.beta, rq, outw);
               break;
             case ACT_SILU:
-              if (has_r) epilogue_chunk<ACT_SILU, true>(accv, bias_s, p.alpha, p.beta, rq, row_addr, lane);
-              else epilogue_chunk<ACT_SILU, false>(accv, bias_s, p.alpha, p.beta, rq, row_addr, lane);
+              if (has_r) epilogue_chunk<ACT_SILU, true>(accv, bias_s, p.alpha, p.beta, rq, outw);
+              else epilogue_chunk<ACT_SILU, false>(accv, bias_s, p.alpha, p.beta, rq, outw);
               break;
             default:
-              if (has_r) epilogue_chunk<ACT_NONE, true>(accv, bias_s, p.alpha, p.beta, rq, row_addr, lane);
-              else epilogue_chunk<ACT_NONE, false>(accv, bias_s, p.alpha, p.beta, rq, row_addr, lane);
+              if (has_r) epilogue_chunk<ACT_NONE, true>(accv, bias_s, p.alpha, p.beta, rq, outw);
+              else epilogue_chunk<ACT_NONE, false>(accv, bias_s, p.alpha, p.beta, rq, outw);
               break;
           }
+          // staging buffer free again?  (the store that last used it has finished reading it) --
+          // asked only now, after the arithmetic, so that the wait overlaps it
+          if (lane == 0) ptx::bulk_wait_group_read<C::EPI_BUFS - 1>();
+          __syncwarp();
+          const uint32_t buf_addr = stage_base + store_buf * EPI_BUF_BYTES;
+          stage_chunk(outw, buf_addr + lane * 128, lane);
           ptx::fence_proxy_async_smem();      // my generic-proxy writes -> visible to the TMA store
           __syncwarp();
           if (lane == 0) {
