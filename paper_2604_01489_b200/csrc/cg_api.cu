@@ -83,18 +83,18 @@ int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
 // ---- kernel table ------------------------------------------------------------------
 
-typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const KernelParams);
+typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const KernelParams);
 
 struct KernelEntry {
   KernelFn fn;
-  int stage_bytes, fixed_bytes, stages_max, threads, sub_cols;
+  int stage_bytes, fixed_bytes, r_bytes, stages_max, stages_max_r, threads, sub_cols;
 };
 
 template <int BN, int CGN, bool KM>
 KernelEntry entry() {
   using C = Cfg<BN, CGN, KM>;
-  return KernelEntry{gemm_epilogue_kernel<BN, CGN, KM>, C::STAGE_BYTES, C::FIXED_BYTES, C::STAGES_MAX, C::NUM_THREADS,
-                     C::SUB_COLS};
+  return KernelEntry{gemm_epilogue_kernel<BN, CGN, KM>, C::STAGE_BYTES, C::FIXED_BYTES, C::R_BYTES, C::stages_max(false),
+                     C::stages_max(true), C::NUM_THREADS, C::SUB_COLS};
 }
 
 // index: [bn_idx (64,128,256)][cg-1][b_kmajor]
@@ -148,7 +148,7 @@ size_t partial_need(long long split_units, int bn, int cgn) {
   return static_cast<size_t>(2) * split_units * cgn * BM * bn * sizeof(float);
 }
 
-int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, Plan* pl) {
+int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, bool has_r, Plan* pl) {
   const cg_tuning_t& t = h->tuning;
   const int sms = (t.max_ctas > 0 && t.max_ctas < h->num_sms) ? t.max_ctas : h->num_sms;
   const int k_blocks = ceil_div(K, BK);
@@ -171,7 +171,8 @@ int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, Plan
         const int pairs = sms / 2 > 0 ? sms / 2 : 1;
         auto eff = [&](long long nt) { return static_cast<double>(nt) / (static_cast<double>((nt + pairs - 1) / pairs) * pairs); };
         const long long t256 = tiles(2 * BM, 256), t512 = tiles(2 * BM, 512);
-        if (t512 >= 2 * pairs && eff(t512) >= eff(t256) - 0.03) bn = 512;
+        // (with a residual the wide tile would be left with three ring stages: not worth it)
+        if (!has_r && t512 >= 2 * pairs && eff(t512) >= eff(t256) - 0.03) bn = 512;
       }
     } else {
       // widest tile that still gives every SM a tile; otherwise the narrowest
@@ -239,11 +240,12 @@ int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, Plan
   pl->num_workers = pl->num_units < max_workers ? pl->num_units : max_workers;
   pl->grid = pl->num_workers * cgn;
 
-  int stages = t.stages > 0 ? t.stages : e.stages_max;
-  if (stages > e.stages_max) stages = e.stages_max;
+  const int smax = has_r ? e.stages_max_r : e.stages_max;       // the residual's chunk buffers cost ring depth
+  int stages = t.stages > 0 ? t.stages : smax;
+  if (stages > smax) stages = smax;
   if (stages < 1) stages = 1;
   pl->stages = stages;
-  pl->smem = stages * e.stage_bytes + e.fixed_bytes + 1024;     // layout + alignment slack, capped at the limit
+  pl->smem = stages * e.stage_bytes + e.fixed_bytes + (has_r ? e.r_bytes : 0) + 1024;   // layout + alignment slack, capped
   if (pl->smem > SMEM_LIMIT) pl->smem = SMEM_LIMIT;
 
   int gm = t.group_m > 0 ? t.group_m : (bn == 512 ? 16 : 8);
@@ -279,17 +281,18 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
            int batch, float alpha, float beta, int act, cudaStream_t stream) {
   const bool b_kmajor = (act & CG_FLAG_B_COLMAJOR) != 0;
   Plan pl;
-  int rc = make_plan(h, M, N, K, batch, b_kmajor, &pl);
+  int rc = make_plan(h, M, N, K, batch, b_kmajor, beta != 0.0f, &pl);
   if (rc != CG_OK) return rc;
   KernelEntry e;
   lookup(pl.bn, pl.cg, b_kmajor, &e);
 
-  CUtensorMap tmA, tmB, tmD;
+  CUtensorMap tmA, tmB, tmD, tmR;
   if ((rc = make_map(h, &tmA, A, K, M, batch, BK, BM)) != CG_OK) return rc;
   if (b_kmajor) rc = make_map(h, &tmB, B, K, N, batch, BK, e.sub_cols);
   else rc = make_map(h, &tmB, B, N, K, batch, 64, BK);
   if (rc != CG_OK) return rc;
   if ((rc = make_map(h, &tmD, D, N, M, batch, EPI_COLS, 32)) != CG_OK) return rc;
+  if ((rc = make_map(h, &tmR, beta != 0.0f ? R : D, N, M, batch, EPI_COLS, 32)) != CG_OK) return rc;   // unused without a residual
 
   KernelParams p;
   memset(&p, 0, sizeof p);
@@ -329,7 +332,7 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  void* args[4] = {&tmA, &tmB, &tmD, &p};
+  void* args[5] = {&tmA, &tmB, &tmD, &tmR, &p};
   CG_CUDA(h, cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(e.fn), args));
 
   cg_plan_info_t& lp = h->last_plan;

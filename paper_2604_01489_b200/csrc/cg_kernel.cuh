@@ -47,7 +47,7 @@ namespace cg {
 constexpr int BM = 128;          // accumulator rows per CTA (TMEM lanes)
 constexpr int BK = 64;           // k-block: 64 bf16 = one 128-byte swizzle row
 constexpr int UMMA_K = 16;       // K of one tcgen05.mma for 16-bit inputs
-constexpr int MAX_STAGES = 12;
+constexpr int MAX_STAGES = 8;
 constexpr int SMEM_LIMIT = 232448;  // 227 KiB opt-in maximum per CTA
 constexpr int EPI_COLS = 64;        // columns per epilogue chunk (one 128-byte bf16 row)
 constexpr int EPI_BUF_BYTES = 32 * EPI_COLS * 2;   // one warp's staging buffer: 32 rows x 128 B
@@ -101,15 +101,17 @@ struct Cfg {
   static constexpr int NUM_THREADS = 64 + 32 * EPI_WARPS;
   static constexpr int EPI_BYTES = EPI_WARPS * EPI_BUFS * EPI_BUF_BYTES;
   static constexpr int BIAS_BYTES = EPI_WARPS * EPI_COLS * 4;   // per warp: one chunk of fp32 bias
-  static constexpr int FIXED_BYTES = EPI_BYTES + BIAS_BYTES + CTRL_BYTES;
+  static constexpr int R_BYTES = EPI_WARPS * EPI_BUF_BYTES;      // per warp: one 64-column chunk of the residual
+  static constexpr int FIXED_BYTES = EPI_BYTES + BIAS_BYTES + CTRL_BYTES;   // + R_BYTES when there is a residual
   // Up to 1023 bytes go to aligning the ring; the kernel checks that what is left suffices.
-  static constexpr int MAX_FIT = (SMEM_LIMIT - FIXED_BYTES) / STAGE_BYTES;
-  static constexpr int STAGES_MAX = MAX_FIT < MAX_STAGES ? MAX_FIT : MAX_STAGES;
+  __host__ __device__ static constexpr int stages_max(bool with_r) {
+    const int fit = (SMEM_LIMIT - FIXED_BYTES - (with_r ? R_BYTES : 0)) / STAGE_BYTES;
+    return fit < MAX_STAGES ? fit : MAX_STAGES;
+  }
   static constexpr int TMEM_COLS = ACC_BUFS * BN <= 32 ? 32 : (ACC_BUFS * BN <= 64 ? 64 : (ACC_BUFS * BN <= 128 ? 128 : (ACC_BUFS * BN <= 256 ? 256 : 512)));
   static constexpr uint32_t IDESC = ptx::instr_desc_bf16(BM * CG, MMA_N, !B_KMAJOR);
-  __host__ __device__ static constexpr int layout_bytes(int stages) { return stages * STAGE_BYTES + FIXED_BYTES; }
-  __host__ __device__ static constexpr int smem_bytes(int stages) {      // request: the layout plus alignment slack, capped at the limit
-    return layout_bytes(stages) + 1024 < SMEM_LIMIT ? layout_bytes(stages) + 1024 : SMEM_LIMIT;
+  __host__ __device__ static constexpr int layout_bytes(int stages, bool with_r) {
+    return stages * STAGE_BYTES + FIXED_BYTES + (with_r ? R_BYTES : 0);
   }
 };
 
@@ -119,6 +121,7 @@ struct Ctrl {
   uint64_t acc_full[2];
   uint64_t acc_empty[2];
   uint64_t drain;
+  uint64_t r_full[8];     // per epilogue warp: its residual chunk has landed
   uint32_t tmem_base;
   int abort;
 };
@@ -269,7 +272,8 @@ __device__ __forceinline__ void stage_chunk(const uint32_t (&out)[EPI_COLS / 2],
 template <int BN, int CG, bool B_KMAJOR>
 __global__ void __launch_bounds__((Cfg<BN, CG, B_KMAJOR>::NUM_THREADS), 1)
 gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                     const __grid_constant__ CUtensorMap tmD, const KernelParams p) {
+                     const __grid_constant__ CUtensorMap tmD, const __grid_constant__ CUtensorMap tmR,
+                     const KernelParams p) {
   using C = Cfg<BN, CG, B_KMAJOR>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = ptx::smem_u32(smem_raw);
@@ -279,12 +283,15 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   const int stages = p.stages;
   uint8_t* epi_ptr = smem + stages * C::STAGE_BYTES;
   const uint32_t epi_addr = ring_addr + stages * C::STAGE_BYTES;
-  float* bias_all = reinterpret_cast<float*>(epi_ptr + C::EPI_BYTES);
-  Ctrl* ctrl = reinterpret_cast<Ctrl*>(epi_ptr + C::EPI_BYTES + C::BIAS_BYTES);
+  const bool has_r = (p.beta != 0.0f);
+  const int r_bytes = has_r ? C::R_BYTES : 0;           // residual chunks sit between the staging buffers and the bias
+  const uint32_t rbuf_addr = epi_addr + C::EPI_BYTES;
+  float* bias_all = reinterpret_cast<float*>(epi_ptr + C::EPI_BYTES + r_bytes);
+  Ctrl* ctrl = reinterpret_cast<Ctrl*>(epi_ptr + C::EPI_BYTES + r_bytes + C::BIAS_BYTES);
   {
     uint32_t dyn_bytes;
     asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn_bytes));
-    if (pad + static_cast<uint32_t>(C::layout_bytes(stages)) > dyn_bytes) {   // never expected: the ring would not fit
+    if (pad + static_cast<uint32_t>(C::layout_bytes(stages, has_r)) > dyn_bytes) {   // never expected: the ring would not fit
       if (threadIdx.x == 0) atomicCAS(p.status, STATUS_OK, STATUS_SMEM);
       return;
     }
@@ -306,6 +313,8 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       ptx::mbar_init(ptx::smem_u32(&ctrl->acc_empty[a]), C::EPI_WARPS * CG);   // one arrive per epilogue warp of the pair
     }
     ptx::mbar_init(ptx::smem_u32(&ctrl->drain), 1);
+    for (int w = 0; w < 8; ++w) ptx::mbar_init(ptx::smem_u32(&ctrl->r_full[w]), 1);
+    ptx::prefetch_tensormap(&tmR);
     ctrl->abort = 0;
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&tmA);
@@ -493,7 +502,20 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     WorkIter wi(p, worker);
     Segment s;
     bool ok = true;
-    const bool has_r = (p.beta != 0.0f);
+    // The residual reaches the epilogue through TMA: one 64-column chunk (32 rows x 128 B, same box
+    // and swizzle as the output staging) per warp, requested one chunk -- and across tiles one
+    // tile -- ahead of its use, so that the reads are coalesced and off the critical path.
+    const uint32_t rbuf = rbuf_addr + ew * EPI_BUF_BYTES;
+    const uint32_t r_bar = ptx::smem_u32(&ctrl->r_full[ew]);
+    uint32_t r_phase = 0;
+    bool r_pending = false;          // a chunk has been requested and not yet read
+    auto request_residual = [&](int col, int row0, int bb) {
+      if (lane == 0) {
+        ptx::mbar_arrive_expect_tx(r_bar, EPI_BUF_BYTES);
+        ptx::tma_load_3d(rbuf, &tmR, r_bar, col, row0, bb);     // outside the tensor: zero fill, same byte count
+      }
+      r_pending = true;
+    };
     // Pulls this thread's row of a tile's residual (its share of the columns) into L2.
     auto prefetch_residual = [&](const Segment& sg) {
       int pb, pmt, pnt;
@@ -513,19 +535,26 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       if (peek.next(s0)) prefetch_residual(s0);
     }
     while (ok && wi.next(s)) {
+      Segment s_next;
+      bool have_next = false;
       if (has_r) {               // the tile after this one: a whole main loop ahead of its use
         WorkIter peek = wi;
-        Segment s1;
-        if (peek.next(s1)) prefetch_residual(s1);
+        have_next = peek.next(s_next);
+        if (have_next) prefetch_residual(s_next);
       }
       int b, mt, nt;
       decode_tile(p, s.tile, b, mt, nt);
       const int m_base = mt * (BM * CG) + static_cast<int>(cta_rank) * BM;   // first row of this CTA's slab
       const int n_base = nt * BN;
-      const int m = m_base + row_in_tile;
-      const bool row_valid = m < p.M;
       const bool warp_rows_valid = (m_base + q * 32) < p.M;
       const bool whole_tile = (s.kb0 == 0 && s.kb1 == p.k_blocks);
+      int n_chunks = (p.N - n_base + EPI_COLS - 1) / EPI_COLS;    // chunks with at least one valid column
+      if (n_chunks > BN / EPI_COLS) n_chunks = BN / EPI_COLS;
+      const int c_lo = col_group * CHUNKS_PER_GROUP;               // this warp's chunk range [c_lo, c_hi)
+      int c_hi = c_lo + CHUNKS_PER_GROUP;
+      if (c_hi > n_chunks) c_hi = n_chunks;
+      if (has_r && whole_tile && !r_pending && c_lo < c_hi)
+        request_residual(n_base + c_lo * EPI_COLS, m_base + q * 32, b);
       // bias of this warp's columns: two values per lane and chunk, fetched before the wait for the
       // accumulator so that the loads are off the critical path
       float bias_reg[2 * CHUNKS_PER_GROUP];
@@ -552,11 +581,6 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(acc * BN);
       const uint32_t acc_empty_bar = (CG == 2) ? ptx::mapa(ptx::smem_u32(&ctrl->acc_empty[acc]), 0)
                                                : ptx::smem_u32(&ctrl->acc_empty[acc]);
-      int n_chunks = (p.N - n_base + EPI_COLS - 1) / EPI_COLS;    // chunks with at least one valid column
-      if (n_chunks > BN / EPI_COLS) n_chunks = BN / EPI_COLS;
-      const int c_lo = col_group * CHUNKS_PER_GROUP;               // this warp's chunk range [c_lo, c_hi)
-      int c_hi = c_lo + CHUNKS_PER_GROUP;
-      if (c_hi > n_chunks) c_hi = n_chunks;
 
       bool reduce = false;        // this warp must run the epilogue from workspace partials
       int first_unit = 0, last_unit = 0;
@@ -597,7 +621,10 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         first_unit = __shfl_sync(0xFFFFFFFFu, first_unit, 0);
         last_unit = __shfl_sync(0xFFFFFFFFu, last_unit, 0);
         reduce = (last != 0);
-        if (reduce) __threadfence();
+        if (reduce) {
+          __threadfence();
+          if (has_r && c_lo < c_hi) request_residual(n_base + c_lo * EPI_COLS, m_base + q * 32, b);
+        }
       }
 
       if (whole_tile || reduce) {
@@ -606,15 +633,6 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           int n_valid = p.N - n0;
           if (n_valid > EPI_COLS) n_valid = EPI_COLS;
           const float bv0 = bias_reg[2 * (c - c_lo)], bv1 = bias_reg[2 * (c - c_lo) + 1];   // fetched at tile start
-          // residual for this chunk: issued now so that its latency overlaps the accumulator read
-          uint4 rq[EPI_COLS / 8];
-          if (has_r) {
-            const uint4* r_row = reinterpret_cast<const uint4*>(
-                p.R + (static_cast<size_t>(b) * p.M + (row_valid ? m : 0)) * p.N + n0);
-#pragma unroll
-            for (int j = 0; j < EPI_COLS / 8; ++j)
-              rq[j] = (row_valid && j * 8 < n_valid) ? r_row[j] : make_uint4(0u, 0u, 0u, 0u);
-          }
           float accv[EPI_COLS];
           if (whole_tile) {
             uint32_t v0[32], v1[32];
@@ -643,6 +661,29 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 const float4 t = __ldcg(part + (c * (EPI_COLS / 4) + j) * 32 + lane);
                 accv[4 * j] += t.x; accv[4 * j + 1] += t.y; accv[4 * j + 2] += t.z; accv[4 * j + 3] += t.w;
               }
+            }
+          }
+          // residual of this chunk: this thread's row of the TMA-filled buffer (swizzled like the staging)
+          uint4 rq[EPI_COLS / 8];
+          if (has_r) {
+            if (!wait_bar(r_bar, r_phase, ctrl, p)) { ok = false; break; }
+            r_phase ^= 1u;
+            r_pending = false;
+#pragma unroll
+            for (int j = 0; j < EPI_COLS / 8; ++j) {
+              const uint32_t addr = rbuf + lane * 128 + (static_cast<uint32_t>(j ^ (lane & 7)) << 4);
+              asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                           : "=r"(rq[j].x), "=r"(rq[j].y), "=r"(rq[j].z), "=r"(rq[j].w) : "r"(addr) : "memory");
+            }
+            __syncwarp();        // every lane has read the buffer: it may be refilled
+            if (c + 1 < c_hi) {
+              request_residual(n0 + EPI_COLS, m_base + q * 32, b);
+            } else if (have_next && s_next.kb0 == 0 && s_next.kb1 == p.k_blocks) {
+              // first chunk of the next whole tile, a main loop ahead
+              int nb2, nmt, nnt;
+              decode_tile(p, s_next.tile, nb2, nmt, nnt);
+              if (nnt * BN + c_lo * EPI_COLS < p.N)
+                request_residual(nnt * BN + c_lo * EPI_COLS, nmt * (BM * CG) + static_cast<int>(cta_rank) * BM + q * 32, nb2);
             }
           }
           bias_s[lane] = bv0;
@@ -690,6 +731,11 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         }
       }
       if (++acc == C::ACC_BUFS) { acc = 0; acc_phase ^= 1u; }
+    }
+    if (r_pending) {                            // (only when leaving early) let the requested chunk land
+      const long long t0 = clock64();
+      while (!ptx::mbar_try_wait(r_bar, r_phase))
+        if (clock64() - t0 > (1ll << 27)) break;
     }
     if (lane == 0) ptx::bulk_wait_group<0>();   // all of this warp's stores have completed
     __syncwarp();
