@@ -38,6 +38,24 @@ struct StagingBuf {
   size_t cap = 0;
 };
 
+// Encoded tensor maps are pure functions of (address, extents, box): a small cache keeps the
+// host cost of repeated calls on the same tensors (the common case) to a few lookups.
+struct MapKey {
+  const void* base;
+  uint64_t inner, rows, batch;
+  uint32_t box_inner, box_rows;
+  bool operator==(const MapKey& o) const {
+    return base == o.base && inner == o.inner && rows == o.rows && batch == o.batch && box_inner == o.box_inner &&
+           box_rows == o.box_rows;
+  }
+};
+struct MapCacheEntry {
+  MapKey key{};
+  CUtensorMap map;
+  bool valid = false;
+};
+constexpr int MAP_CACHE_SIZE = 16;
+
 }  // namespace
 
 struct cg_context {
@@ -56,6 +74,9 @@ struct cg_context {
   char last_msg[256] = {0};
   long long wait_limit = 4000000000ll;   // about two seconds of SM clocks
   int test_starve = 0;                   // test hook (CG_TEST_STARVE): see KernelParams::test_starve
+  bool log_plans = false;                // CG_LOG
+  MapCacheEntry map_cache[MAP_CACHE_SIZE];
+  int map_cache_next = 0;
   StagingBuf sA, sB, sBias, sR, sD;
   std::mutex mu;
 };
@@ -129,6 +150,12 @@ int prepare_kernels(cg_context* h) {
 // bf16, rank 3 (inner, rows, batch), 128-byte swizzle, zero fill outside the tensor.
 int make_map(cg_context* h, CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows, uint64_t batch,
              uint32_t box_inner, uint32_t box_rows) {
+  const MapKey key{base, inner, rows, batch, box_inner, box_rows};
+  for (int i = 0; i < MAP_CACHE_SIZE; ++i)
+    if (h->map_cache[i].valid && h->map_cache[i].key == key) {
+      *map = h->map_cache[i].map;
+      return CG_OK;
+    }
   const cuuint64_t dims[3] = {inner, rows, batch};
   const cuuint64_t strides[2] = {inner * 2, inner * rows * 2};
   const cuuint32_t box[3] = {box_inner, box_rows, 1};
@@ -139,6 +166,11 @@ int make_map(cg_context* h, CUtensorMap* map, const void* base, uint64_t inner, 
   if (r != CUDA_SUCCESS)
     return fail(h, CG_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d) for dims %llu x %llu x %llu box %u x %u", (int)r,
                 (unsigned long long)inner, (unsigned long long)rows, (unsigned long long)batch, box_inner, box_rows);
+  MapCacheEntry& slot = h->map_cache[h->map_cache_next];
+  h->map_cache_next = (h->map_cache_next + 1) % MAP_CACHE_SIZE;
+  slot.key = key;
+  slot.map = *map;
+  slot.valid = true;
   return CG_OK;
 }
 
@@ -342,7 +374,7 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   lp.smem_bytes = pl.smem; lp.launches = 1;
   h->last_status = CG_OK;
   h->last_msg[0] = 0;
-  if (getenv("CG_LOG"))
+  if (h->log_plans)
     fprintf(stderr, "[cg] M=%d N=%d K=%d batch=%d tile=%dx%d cg=%d stages=%d group_m=%d grid=%d tiles=%d units=%d smem=%d\n", M,
             N, K, batch, lp.tile_m, lp.tile_n, lp.cta_group, lp.stages, lp.group_m, lp.grid, lp.num_tiles, lp.num_units,
             lp.smem_bytes);
@@ -405,6 +437,7 @@ int cg_create(cg_handle_t* out, int device, size_t workspace_bytes) {
     if (v > 0) h->wait_limit = v;
   }
   if (const char* w = getenv("CG_TEST_STARVE")) h->test_starve = atoi(w) != 0;
+  h->log_plans = getenv("CG_LOG") != nullptr;
   *out = h;
   return CG_OK;
 }
