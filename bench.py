@@ -156,6 +156,25 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# ------------------------------------------------------------------ multi-rank arithmetic
+
+def max_over_ranks(values, device=None):
+    """Element-wise MAX of a list of floats over all ranks of the default process group (identity
+    when there is none): a multi-GPU time is the slowest rank's."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor(values, dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_tflops(flops_per_step: float, steps: int, world: int, seconds: float) -> float:
+    """Every rank runs its own replica of the workload: the job's work is world x one rank's."""
+    return world * flops_per_step * steps / seconds / 1e12
+
+
 # ------------------------------------------------------------------ our arm
 
 def to_device(p, device):
@@ -179,23 +198,103 @@ def pinned(x):
 def per_launch_times(ctx, p, dev, iters, flush):
     """Each launch timed alone with CUDA events on the launching stream; L2 flushed in between."""
     import torch
-    ts = []
+    evs = []
     for _ in range(iters):
         if flush is not None:
-            flush.fill_(1)
+            flush.fill_(1)       # also gives the host time to enqueue the launch: no host gap is timed
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         ctx.gemm_epilogue(dev["A"], dev["B"], dev["bias"], dev["R"], dev["D"], p.M, p.N, p.K, p.batch, p.alpha, p.beta, p.act)
         e1.record()
+        evs.append((e0, e1))
+    torch.cuda.synchronize()
+    return [a.elapsed_time(b) * 1e-3 for a, b in evs]
+
+
+def timed(fn, iters, flush):
+    """fn() timed launch by launch with CUDA events on the current stream, L2 flushed before each."""
+    import torch
+    evs = []
+    for _ in range(iters):
+        flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        evs.append((e0, e1))
+    torch.cuda.synchronize()
+    return [a.elapsed_time(b) * 1e-3 for a, b in evs]
+
+
+def library_side_by_side(p, dev, flush):
+    """Timing only, never on the hot path: cuBLAS through torch.bmm (GEMM alone) and the unfused
+    PyTorch-eager form of the whole expression (the paper's comparison convention)."""
+    import torch
+    import torch.nn.functional as F
+    A, B, D = dev["A"], dev["B"], dev["D"]
+    Bm = B.transpose(1, 2) if p.act & W.FLAG_B_COLMAJOR else B
+    kind = p.act & 0xFF
+
+    def eager():
+        t = torch.bmm(A, Bm)
+        if p.alpha != 1.0:
+            t = t * p.alpha
+        if dev["bias"] is not None:
+            t = t + dev["bias"].to(t.dtype)
+        if kind == W.ACT_RELU:
+            t = torch.relu(t)
+        elif kind == W.ACT_GELU_TANH:
+            t = F.gelu(t, approximate="tanh")
+        elif kind == W.ACT_SILU:
+            t = F.silu(t)
+        if p.beta != 0.0:
+            t = t + p.beta * dev["R"]
+        return t
+
+    out = {}
+    for key, fn in (("cublas_gemm_only_us_best", lambda: torch.bmm(A, Bm, out=D)), ("torch_eager_unfused_us_best", eager)):
+        timed(fn, 3, flush)
+        out[key] = min(timed(fn, 10, flush)) * 1e6
+    return out
+
+
+def small_problem_extras(ctx, p, dev, flush):
+    """Latency-bound workload: the same launch replayed from a CUDA graph (no host in the loop, inputs
+    warm in L2) and the floor of the measurement itself (a one-element fill kernel)."""
+    import torch
+    call = lambda: ctx.gemm_epilogue(dev["A"], dev["B"], dev["bias"], dev["R"], dev["D"], p.M, p.N, p.K, p.batch, p.alpha,
+                                     p.beta, p.act)
+    reps = 20
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        call()
+    torch.cuda.current_stream().wait_stream(side)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for _ in range(reps):
+            call()
+    graph.replay()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(10):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        graph.replay()
+        e1.record()
         e1.synchronize()
-        ts.append(e0.elapsed_time(e1) * 1e-3)
-    return ts
+        ts.append(e0.elapsed_time(e1) * 1e-3 / reps)
+    one = torch.zeros(1, device=dev["D"].device)
+    floor = min(timed(lambda: one.fill_(1.0), 20, flush))
+    return {"us_graph_replay_per_launch": min(ts) * 1e6, "us_measurement_floor_one_element_fill": floor * 1e6}
 
 
 def workload_table(ctx, device, peaks, names):
-    """All five workloads, each launch timed alone after an L2 flush (their inputs may fit in L2)."""
+    """All five workloads under the heuristic plan, each launch timed alone after an L2 flush (their
+    inputs may fit in L2)."""
     import torch
     flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=device)
+    ctx.set_tuning(reset=True)
     out = {}
     for name in names:
         p = W.config(name)
@@ -210,6 +309,9 @@ def workload_table(ctx, device, peaks, names):
                "frac_tensor_of_nominal_2250": p.flops / best / 1e12 / 2250.0,
                "frac_hbm_of_measured": p.algorithmic_bytes / best / 1e9 / peaks["hbm_gbs"],
                "bound": BOUND[name], "plan": ctx.last_plan()}
+        row.update(library_side_by_side(p, dev, flush))
+        if BOUND[name] == "latency":
+            row.update(small_problem_extras(ctx, p, dev, flush))
         out[name] = row
         del dev
     return out
@@ -239,6 +341,10 @@ def run_ours(args):
     p = W.config(args.config)                      # seeded host buffers (the same ones the oracle would read)
     dev = to_device(p, device)
     ctx = cg.Context(local_rank)
+    tuning = dict(tile_n=args.tile_n, cta_group=args.cta_group, num_units=args.num_units, dp_units=args.dp_units,
+                  stages=args.stages, group_m=args.group_m, max_ctas=args.max_ctas)
+    if any(tuning.values()):
+        ctx.set_tuning(**tuning)
     launch = lambda: ctx.gemm_epilogue(dev["A"], dev["B"], dev["bias"], dev["R"], dev["D"], p.M, p.N, p.K, p.batch,
                                        p.alpha, p.beta, p.act)
     footprint = p.algorithmic_bytes
@@ -287,13 +393,9 @@ def run_ours(args):
         h2d = p.A.nbytes + p.B.nbytes + (p.bias.nbytes if p.bias is not None else 0) + (p.R.nbytes if hR is not None else 0)
         d2h = hD.numel() * 2
 
-    if world > 1:
-        t = torch.tensor([total_s, e2e_s], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_s, e2e_s = float(t[0]), float(t[1])
-
-    value = world * p.flops * args.steps / total_s / 1e12
-    e2e_value = world * p.flops * e2e_steps / e2e_s / 1e12
+    total_s, e2e_s = max_over_ranks([total_s, e2e_s], device)
+    value = whole_job_tflops(p.flops, args.steps, world, total_s)
+    e2e_value = whole_job_tflops(p.flops, e2e_steps, world, e2e_s)
     per_launch_s = total_s / args.steps
     bound = BOUND[args.config]
     if bound == "hbm":
@@ -343,6 +445,8 @@ def main():
     ap.add_argument("--config", default=DEFAULT_CONFIG, choices=W.CONFIG_ORDER)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-table", action="store_true", help="skip the five-workload table")
+    for flag in ("tile-n", "cta-group", "num-units", "dp-units", "stages", "group-m", "max-ctas"):
+        ap.add_argument(f"--{flag}", type=int, default=0, help="plan override for ablations (0 = heuristic)")
     ap.add_argument("--kernel-only", action="store_true",
                     help="only the device-timed region (for profiler runs): no e2e, no CPU baseline, no table")
     args = ap.parse_args()

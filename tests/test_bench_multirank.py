@@ -1,0 +1,65 @@
+"""The multi-rank side of bench.py on CPU (gloo, world size 2): the max-over-ranks reduction, the
+whole-job arithmetic, and the reference arm under torchrun (rank 0 alone works and prints)."""
+import json
+import os
+import socket
+import subprocess
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+WORKER = r"""
+import os, sys
+sys.path.insert(0, {root!r})
+import torch.distributed as dist
+import bench
+dist.init_process_group("gloo")
+rank, world = dist.get_rank(), dist.get_world_size()
+got = bench.max_over_ranks([1.0 + rank, 10.0 - rank, 0.5])
+assert got == [float(world), 10.0, 0.5], got
+assert abs(bench.whole_job_tflops(2e12, 5, world, got[0]) - world * 2e12 * 5 / world / 1e12) < 1e-9
+dist.barrier()
+dist.destroy_process_group()
+sys.stdout.write("RANK_OK_%d\n" % rank)     # one write per rank: the two ranks share a pipe
+"""
+
+
+def test_max_over_ranks_gloo_world2(tmp_path):
+    script = tmp_path / "worker.py"
+    script.write_text(WORKER.format(root=ROOT))
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2", "--master-addr", "127.0.0.1",
+           "--master-port", str(free_port()), str(script)]
+    res = subprocess.run(cmd, capture_output=True, text=True, timeout=300)
+    assert res.returncode == 0, res.stdout + res.stderr
+    assert "RANK_OK_0" in res.stdout and "RANK_OK_1" in res.stdout
+
+
+def test_single_process_identity():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.max_over_ranks([3.0, 4.5]) == [3.0, 4.5]
+    assert bench.whole_job_tflops(1e12, 10, 1, 2.0) == 5.0
+    assert bench.whole_job_tflops(1e12, 10, 8, 2.0) == 40.0
+
+
+def test_reference_arm_under_torchrun_prints_one_line():
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2", "--master-addr", "127.0.0.1",
+           "--master-port", str(free_port()), os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "1",
+           "--warmup", "0", "--config", "cfg1_256_relu"]
+    res = subprocess.run(cmd, capture_output=True, text=True, timeout=600)
+    assert res.returncode == 0, res.stdout + res.stderr
+    lines = [ln for ln in res.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["impl"] == "reference" and d["n_gpus"] == 2 and d["unit"] == "TFLOP/s" and d["value"] > 0
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] == 1
+    assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["vs_baseline"] is None
