@@ -207,9 +207,11 @@ int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, bool
         if (!has_r && t512 >= 2 * pairs && eff(t512) >= eff(t256) - 0.03) bn = 512;
       }
     } else {
-      // widest tile that still gives every SM a tile; otherwise the narrowest
+      // widest tile that still gives every SM a tile; otherwise the narrowest -- except that a
+      // 128-wide tile cut in two along K is preferred to a 64-wide one: an MMA costs the same 128
+      // clocks whatever its N, so halving N doubles the tensor time per byte streamed
       bn = 64;
-      if (N >= 128 && tiles(BM, 128) >= sms) bn = 128;
+      if (N >= 128 && (tiles(BM, 128) >= sms || (K >= 512 && tiles(BM, 128) * 10 >= static_cast<long long>(sms) * 4))) bn = 128;
       if (N >= 256 && tiles(BM, 256) >= sms) bn = 256;
     }
   }
