@@ -105,6 +105,9 @@ typedef struct cg_tuning {
                     anything else -> stream-K (tile_n <= 256)                               */
   int dp_units;  /* with num_units: the first dp_units units are whole tiles, the other
                     num_units - dp_units divide the remaining tiles' iterations evenly      */
+  int cluster_split; /* 1-CTA tiles: 2 or 4 = the CTAs of a cluster hold the K parts of one tile and
+                    reduce them through distributed shared memory (tile_n / parts >= 64,
+                    k-blocks divisible by parts); 1 = never; 0 = heuristic                  */
   int stages;    /* depth of the shared-memory operand ring (clamped to what fits)          */
   int group_m;   /* raster: m-tiles walked before stepping to the next n-tile               */
   int max_ctas;  /* cap on the persistent grid (0 = one CTA per SM)                         */
@@ -121,6 +124,7 @@ typedef struct cg_plan_info {
   int k_blocks;    /* 64-wide k-blocks per tile              */
   int smem_bytes;  /* dynamic shared memory per CTA          */
   int launches;    /* kernels launched by the call (always 1)*/
+  int cluster_split; /* K parts per tile held by one cluster (1 = off) */
 } cg_plan_info_t;
 CG_API int cg_get_last_plan(cg_handle_t h, cg_plan_info_t* out);
 

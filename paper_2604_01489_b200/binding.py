@@ -25,12 +25,12 @@ EXPORTS = ["cg_create", "cg_gemm_epilogue", "cg_gemm_epilogue_host", "cg_set_tun
 
 
 class cg_tuning_t(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_int) for n in ("tile_n", "cta_group", "num_units", "dp_units", "stages", "group_m", "max_ctas")]
+    _fields_ = [(n, ctypes.c_int) for n in ("tile_n", "cta_group", "num_units", "dp_units", "cluster_split", "stages", "group_m", "max_ctas")]
 
 
 class cg_plan_info_t(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in ("tile_m", "tile_n", "cta_group", "stages", "group_m", "grid", "num_tiles",
-                                            "num_units", "dp_units", "k_blocks", "smem_bytes", "launches")]
+                                            "num_units", "dp_units", "k_blocks", "smem_bytes", "launches", "cluster_split")]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}
@@ -136,10 +136,11 @@ def cg_gemm_epilogue_host(h, A, B, bias, R, D, M, N, K, batch, alpha, beta, act,
                                         _stream_ptr(stream))
 
 
-def cg_set_tuning(h, tile_n=0, cta_group=0, num_units=0, dp_units=0, stages=0, group_m=0, max_ctas=0, reset=False) -> int:
+def cg_set_tuning(h, tile_n=0, cta_group=0, num_units=0, dp_units=0, stages=0, group_m=0, max_ctas=0, cluster_split=0,
+                  reset=False) -> int:
     if reset:
         return load().cg_set_tuning(h, None)
-    t = cg_tuning_t(tile_n, cta_group, num_units, dp_units, stages, group_m, max_ctas)
+    t = cg_tuning_t(tile_n, cta_group, num_units, dp_units, cluster_split, stages, group_m, max_ctas)
     return load().cg_set_tuning(h, ctypes.byref(t))
 
 

@@ -28,7 +28,7 @@ constexpr int MAX_TICKET_TILES = 1 << 16;          // (tile, CTA) pairs that may
 constexpr int TICKETS_PER_TILE = 8;                // one ticket per epilogue warp slot
 
 struct Plan {
-  int bn, cg, stages, group_m, num_units, dp_units, grid, num_workers;
+  int bn, cg, stages, group_m, num_units, dp_units, grid, num_workers, cluster_split;
   int tiles_m, tiles_n, num_tiles, k_blocks, smem;
   bool b_kmajor;
 };
@@ -192,7 +192,7 @@ int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, bool
   if (cgn == 0) {
     // CTA pairs halve B's shared-memory traffic per flop; worth it once the machine is full
     const int bn2 = bn ? bn : 256;
-    cgn = (M > BM && N >= 128 && bn2 >= 128 && tiles(2 * BM, bn2) >= sms) ? 2 : 1;
+    cgn = (t.cluster_split <= 1 && M > BM && N >= 128 && bn2 >= 128 && tiles(2 * BM, bn2) >= sms) ? 2 : 1;
   }
   if (bn == 0) {
     if (cgn == 2) {
@@ -213,6 +213,29 @@ int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, bool
       bn = 64;
       if (N >= 128 && (tiles(BM, 128) >= sms || (K >= 512 && tiles(BM, 128) * 10 >= static_cast<long long>(sms) * 4))) bn = 128;
       if (N >= 256 && tiles(BM, 256) >= sms) bn = 256;
+    }
+  }
+  // Problems of under one wave of 1-CTA tiles: split K across the CTAs of a cluster, which exchange
+  // their partial tiles through distributed shared memory.  Wider tiles first (an MMA costs the same
+  // whatever its N, and more of B is in flight per SM); each CTA must own at least 64 columns.
+  int csk = 1;
+  auto csk_ok = [&](int bn_, int parts) {
+    return cgn == 1 && parts >= 2 && parts <= 8 && (parts & (parts - 1)) == 0 && bn_ / parts >= 64 && N >= bn_ &&
+           k_blocks % parts == 0 && k_blocks / parts >= 4;
+  };
+  if (t.cluster_split > 1) {
+    if (bn == 0) bn = 64 * t.cluster_split > 256 ? 256 : (64 * t.cluster_split < 128 ? 128 : 64 * t.cluster_split);
+    if (!csk_ok(bn, t.cluster_split))
+      return fail(h, CG_ERR_UNSUPPORTED, "cluster_split=%d does not fit tile_n=%d, K=%d", t.cluster_split, bn, K);
+    csk = t.cluster_split;
+  } else if (t.cluster_split == 0 && t.tile_n == 0 && t.num_units == 0 && cgn == 1) {
+    const int cand[3][2] = {{256, 4}, {256, 2}, {128, 2}};
+    for (int i = 0; i < 3 && csk == 1; ++i) {
+      const long long ctas = tiles(BM, cand[i][0]) * cand[i][1];
+      if (csk_ok(cand[i][0], cand[i][1]) && ctas <= sms && ctas * 10 >= static_cast<long long>(sms) * 7) {
+        bn = cand[i][0];
+        csk = cand[i][1];
+      }
     }
   }
   KernelEntry e;
@@ -240,7 +263,10 @@ int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, bool
   // a tile count the ticket array covers and partial-tile space in the workspace.
   const bool can_split = bn <= 256 && static_cast<long long>(pl->num_tiles) * cgn <= MAX_TICKET_TILES;
   long long units = pl->num_tiles, dp = pl->num_tiles;
-  if (t.num_units > 0) {
+  if (csk > 1) {
+    units = static_cast<long long>(pl->num_tiles) * csk;     // unit u = (tile u / csk, part u % csk), one per CTA
+    dp = 0;
+  } else if (t.num_units > 0) {
     units = t.num_units;
     dp = t.dp_units;
     if (dp > pl->num_tiles || dp > units) return fail(h, CG_ERR_INVALID_ARG, "dp_units exceeds the tile or unit count");
@@ -263,7 +289,7 @@ int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, bool
   if (split_units > rest) split_units = rest;
   if (split_units < 1 && rest > 0) split_units = 1;
   units = dp + split_units;
-  if (split_units > 0 && split_units != pl->num_tiles - dp) {     // some unit boundary falls inside a tile
+  if (csk == 1 && split_units > 0 && split_units != pl->num_tiles - dp) {     // some unit boundary falls inside a tile
     if (!can_split) return fail(h, CG_ERR_UNSUPPORTED, "this tile shape or tile count cannot be split along K");
     if (partial_need(split_units, bn, cgn) > h->partial_bytes)
       return fail(h, CG_ERR_WORKSPACE, "split plan needs %zu bytes of workspace, handle has %zu",
@@ -272,12 +298,16 @@ int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, bool
   pl->num_units = static_cast<int>(units);
   pl->dp_units = static_cast<int>(dp);
   pl->num_workers = pl->num_units < max_workers ? pl->num_units : max_workers;
+  if (csk > 1) pl->num_workers = pl->num_units;              // not persistent: the cluster is the unit of scheduling
   pl->grid = pl->num_workers * cgn;
+  pl->cluster_split = csk;
 
   const int smax = has_r ? e.stages_max_r : e.stages_max;       // the residual's chunk buffers cost ring depth
   int stages = t.stages > 0 ? t.stages : smax;
   if (stages > smax) stages = smax;
   if (stages < 1) stages = 1;
+  if (csk > 1 && static_cast<long long>(stages) * e.stage_bytes < static_cast<long long>(BM) * bn * 4)
+    return fail(h, CG_ERR_UNSUPPORTED, "cluster split needs a ring of at least %d bytes for the partial tiles", BM * bn * 4);
   pl->stages = stages;
   pl->smem = stages * e.stage_bytes + e.fixed_bytes + (has_r ? e.r_bytes : 0) + 1024;   // layout + alignment slack, capped
   if (pl->smem > SMEM_LIMIT) pl->smem = SMEM_LIMIT;
@@ -342,6 +372,7 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   p.unit_r = split_units > 0 ? static_cast<int>(rest % split_units) : 0;
   p.num_workers = pl.num_workers;
   p.stages = pl.stages;
+  p.cluster_split = pl.cluster_split;
   p.alpha = alpha; p.beta = beta;
   p.act = act & 0xFF;
   p.bias_bf16 = (act & CG_FLAG_BIAS_BF16) ? 1 : 0;
@@ -361,7 +392,7 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = pl.cg;
+  attr[0].val.clusterDim.x = pl.cluster_split > 1 ? pl.cluster_split : pl.cg;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
@@ -373,7 +404,7 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   lp.tile_m = BM * pl.cg; lp.tile_n = pl.bn; lp.cta_group = pl.cg; lp.stages = pl.stages; lp.group_m = pl.group_m;
   lp.grid = pl.grid; lp.num_tiles = pl.num_tiles; lp.num_units = pl.num_units; lp.dp_units = pl.dp_units;
   lp.k_blocks = pl.k_blocks;
-  lp.smem_bytes = pl.smem; lp.launches = 1;
+  lp.smem_bytes = pl.smem; lp.launches = 1; lp.cluster_split = pl.cluster_split;
   h->last_status = CG_OK;
   h->last_msg[0] = 0;
   if (h->log_plans)
@@ -489,7 +520,7 @@ int cg_set_tuning(cg_handle_t h, const cg_tuning_t* t) {
     return CG_OK;
   }
   if ((t->tile_n != 0 && t->tile_n != 64 && t->tile_n != 128 && t->tile_n != 256 && t->tile_n != 512) || t->cta_group < 0 ||
-      t->cta_group > 2 || t->num_units < 0 || t->dp_units < 0 || t->stages < 0 || t->group_m < 0 || t->max_ctas < 0)
+      t->cta_group > 2 || t->cluster_split < 0 || t->cluster_split > 8 || t->num_units < 0 || t->dp_units < 0 || t->stages < 0 || t->group_m < 0 || t->max_ctas < 0)
     return fail(h, CG_ERR_INVALID_ARG, "bad tuning values");
   h->tuning = *t;
   return CG_OK;

@@ -27,6 +27,13 @@
 // 128 rows of A and half of the B columns, the leader CTA issues tcgen05.mma.cta_group::2,
 // each CTA's epilogue drains its own 128 accumulator rows.
 //
+// Cluster split-K (cluster_split = S > 1, 1-CTA tiles, problems of under one wave): the S CTAs of
+// a cluster each accumulate one K part of the same tile; after a cluster barrier every CTA sends
+// the columns CTA d owns (BN / S of them) straight into d's shared memory (the idle operand ring)
+// with st.shared::cluster, a second cluster barrier follows, and every CTA sums its columns in
+// part order and runs the epilogue on them.  No workspace, no tickets, no trip through L2, and the
+// epilogue work is spread over all S CTAs.
+//
 // BN == 512 (CTA pairs only) is the wide form for large compute-bound problems: two N = 256 MMAs
 // per 16-wide k-step share one A operand, which cuts the bytes fetched from L2 per flop by a
 // quarter (the L2-to-SM path, not the tensor pipe, is what stalls the 256 x 256 form).  Its
@@ -67,6 +74,7 @@ struct KernelParams {
   int unit_q, unit_r;     // ... the rest cut the remaining iterations evenly: start = base + v*q + min(v, r)
   int num_workers;        // CTAs (CG == 1) or CTA pairs (CG == 2)
   int stages;
+  int cluster_split;      // > 1: the CTAs of a cluster of this size hold the K parts of one tile (CG == 1 only)
   float alpha, beta;
   int act;
   int bias_bf16;
@@ -414,6 +422,10 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       }
     }
     __syncwarp();
+    if (CG == 1 && p.cluster_split > 1) {      // the epilogue warps exchange partial tiles between these two
+      ptx::cluster_arrive(); ptx::cluster_wait();
+      ptx::cluster_arrive(); ptx::cluster_wait();
+    }
   } else if (warp == 1) {
     // ================================================================ MMA issuer
     // One thread feeds the tensor pipe, so its instruction count per k-block is what bounds
@@ -487,6 +499,10 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       }
     }
     __syncwarp();
+    if (CG == 1 && p.cluster_split > 1) {
+      ptx::cluster_arrive(); ptx::cluster_wait();
+      ptx::cluster_arrive(); ptx::cluster_wait();
+    }
   } else {
     // ================================================================ epilogue (warps 2 and up)
     const int ew = warp - 2;                    // epilogue warp index
@@ -502,6 +518,10 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     WorkIter wi(p, worker);
     Segment s;
     bool ok = true;
+    const int csk = (CG == 1 && p.cluster_split > 1) ? p.cluster_split : 1;   // cluster split-K: parts per tile
+    const int my_part = (csk > 1) ? static_cast<int>(ptx::cluster_ctarank()) : 0;
+    const int slice_cols = BN / csk;             // columns each CTA of the cluster owns in the final reduction
+    int cluster_barriers_done = 0;
     // The residual reaches the epilogue through TMA: one 64-column chunk (32 rows x 128 B, same box
     // and swizzle as the output staging) per warp, requested one chunk -- and across tiles one
     // tile -- ahead of its use, so that the reads are coalesced and off the critical path.
@@ -550,17 +570,24 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       const bool whole_tile = (s.kb0 == 0 && s.kb1 == p.k_blocks);
       int n_chunks = (p.N - n_base + EPI_COLS - 1) / EPI_COLS;    // chunks with at least one valid column
       if (n_chunks > BN / EPI_COLS) n_chunks = BN / EPI_COLS;
-      const int c_lo = col_group * CHUNKS_PER_GROUP;               // this warp's chunk range [c_lo, c_hi)
+      // this warp's chunks: c_lo, c_lo + c_step, ... below c_hi.  Normally a contiguous share of the
+      // tile; with the cluster split, its share of the columns this CTA owns.
+      int c_lo = col_group * CHUNKS_PER_GROUP, c_step = 1;
       int c_hi = c_lo + CHUNKS_PER_GROUP;
+      if (csk > 1) {
+        c_lo = my_part * (slice_cols / EPI_COLS) + col_group;
+        c_step = C::EPI_COL_GROUPS;
+        c_hi = (my_part + 1) * (slice_cols / EPI_COLS);
+      }
       if (c_hi > n_chunks) c_hi = n_chunks;
-      if (has_r && whole_tile && !r_pending && c_lo < c_hi)
+      if (has_r && (whole_tile || csk > 1) && !r_pending && c_lo < c_hi)
         request_residual(n_base + c_lo * EPI_COLS, m_base + q * 32, b);
       // bias of this warp's columns: two values per lane and chunk, fetched before the wait for the
       // accumulator so that the loads are off the critical path
       float bias_reg[2 * CHUNKS_PER_GROUP];
 #pragma unroll
       for (int j = 0; j < CHUNKS_PER_GROUP; ++j) {
-        const int col = n_base + (col_group * CHUNKS_PER_GROUP + j) * EPI_COLS + lane;
+        const int col = n_base + (c_lo + j * c_step) * EPI_COLS + lane;
         float b0 = 0.0f, b1 = 0.0f;
         if (p.bias != nullptr) {
           if (p.bias_bf16) {
@@ -584,7 +611,33 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 
       bool reduce = false;        // this warp must run the epilogue from workspace partials
       int first_unit = 0, last_unit = 0;
-      if (!whole_tile) {
+      if (csk > 1) {
+        // ---- cluster split-K: exchange the partial tiles through distributed shared memory
+        ptx::cluster_arrive();                 // A: every CTA of the cluster is done with its operand ring
+        ptx::cluster_wait();
+        ++cluster_barriers_done;
+        constexpr int GROUPS32 = BN / 32 / C::EPI_COL_GROUPS;
+        for (int c = col_group * GROUPS32; c < (col_group + 1) * GROUPS32; ++c) {
+          uint32_t v[32];
+          ptx::tmem_ld_32x32b_x32(taddr + c * 32, v);
+          ptx::tmem_ld_wait();
+          const int owner = (c * 32) / slice_cols;                    // CTA that finishes these 32 columns
+          const int off4 = (c * 32 - owner * slice_cols) / 4;         // float4 column inside the owner's slice
+          // receive buffer of the owner: [part][float4 column][row], lanes (rows) contiguous
+          const uint32_t dst = ptx::mapa(ring_addr + ((my_part * (slice_cols / 4) + off4) * BM + row_in_tile) * 16,
+                                         static_cast<uint32_t>(owner));
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            ptx::st_cluster_v4(dst + j * (BM * 16), __uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                               __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+        }
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(acc_empty_bar);
+        ptx::cluster_arrive();                 // B: all partial tiles have been delivered
+        ptx::cluster_wait();
+        ++cluster_barriers_done;
+      } else if (!whole_tile) {
         // ---- split tile: park the fp32 partial, draw a ticket
         const int slot = (2 * (s.unit - p.dp_units) + (s.head ? 0 : 1)) * CG + static_cast<int>(cta_rank);
         float4* part = reinterpret_cast<float4*>(p.partials) + (static_cast<size_t>(slot) * (BM * BN / 4)) +
@@ -627,14 +680,26 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         }
       }
 
-      if (whole_tile || reduce) {
-        for (int c = c_lo; c < c_hi; ++c) {
+      if (whole_tile || reduce || csk > 1) {
+        int c_ord = 0;             // position of the chunk in this warp's list
+        for (int c = c_lo; c < c_hi; c += c_step, ++c_ord) {
           const int n0 = n_base + c * EPI_COLS;
-          int n_valid = p.N - n0;
-          if (n_valid > EPI_COLS) n_valid = EPI_COLS;
-          const float bv0 = bias_reg[2 * (c - c_lo)], bv1 = bias_reg[2 * (c - c_lo) + 1];   // fetched at tile start
+          const float bv0 = bias_reg[2 * c_ord], bv1 = bias_reg[2 * c_ord + 1];   // fetched at tile start
           float accv[EPI_COLS];
-          if (whole_tile) {
+          if (csk > 1) {
+            // sum the parts in part order (deterministic) from this CTA's receive buffer
+#pragma unroll
+            for (int j = 0; j < EPI_COLS; ++j) accv[j] = 0.0f;
+            const int off4 = (c * EPI_COLS - my_part * slice_cols) / 4;
+            for (int src = 0; src < csk; ++src) {
+              const float4* rb = reinterpret_cast<const float4*>(smem) + (src * (slice_cols / 4) + off4) * BM + row_in_tile;
+#pragma unroll
+              for (int j = 0; j < EPI_COLS / 4; ++j) {
+                const float4 t = rb[j * BM];
+                accv[4 * j] += t.x; accv[4 * j + 1] += t.y; accv[4 * j + 2] += t.z; accv[4 * j + 3] += t.w;
+              }
+            }
+          } else if (whole_tile) {
             uint32_t v0[32], v1[32];
             ptx::tmem_ld_32x32b_x32(taddr + c * EPI_COLS, v0);
             ptx::tmem_ld_32x32b_x32(taddr + c * EPI_COLS + 32, v1);
@@ -676,8 +741,8 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                            : "=r"(rq[j].x), "=r"(rq[j].y), "=r"(rq[j].z), "=r"(rq[j].w) : "r"(addr) : "memory");
             }
             __syncwarp();        // every lane has read the buffer: it may be refilled
-            if (c + 1 < c_hi) {
-              request_residual(n0 + EPI_COLS, m_base + q * 32, b);
+            if (c + c_step < c_hi) {
+              request_residual(n0 + c_step * EPI_COLS, m_base + q * 32, b);
             } else if (have_next && s_next.kb0 == 0 && s_next.kb1 == p.k_blocks) {
               // first chunk of the next whole tile, a main loop ahead
               int nb2, nmt, nnt;
@@ -731,6 +796,10 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         }
       }
       if (++acc == C::ACC_BUFS) { acc = 0; acc_phase ^= 1u; }
+    }
+    for (; csk > 1 && cluster_barriers_done < 2; ++cluster_barriers_done) {   // (only when leaving early)
+      ptx::cluster_arrive();
+      ptx::cluster_wait();
     }
     if (r_pending) {                            // (only when leaving early) let the requested chunk land
       const long long t0 = clock64();
