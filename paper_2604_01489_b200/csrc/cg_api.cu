@@ -220,7 +220,7 @@ int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, bool
   // whatever its N, and more of B is in flight per SM); each CTA must own at least 64 columns.
   int csk = 1;
   auto csk_ok = [&](int bn_, int parts) {
-    return cgn == 1 && parts >= 2 && parts <= 8 && (parts & (parts - 1)) == 0 && bn_ / parts >= 64 && N >= bn_ &&
+    return cgn == 1 && (parts == 2 || parts == 4) && bn_ / parts >= 64 && N >= bn_ &&
            k_blocks % parts == 0 && k_blocks / parts >= 4;
   };
   if (t.cluster_split > 1) {
@@ -229,7 +229,7 @@ int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, bool
       return fail(h, CG_ERR_UNSUPPORTED, "cluster_split=%d does not fit tile_n=%d, K=%d", t.cluster_split, bn, K);
     csk = t.cluster_split;
   } else if (t.cluster_split == 0 && t.tile_n == 0 && t.num_units == 0 && cgn == 1) {
-    const int cand[3][2] = {{256, 4}, {256, 2}, {128, 2}};
+    const int cand[3][2] = {{128, 2}, {256, 4}, {256, 2}};     // measured order on the skinny workload
     for (int i = 0; i < 3 && csk == 1; ++i) {
       const long long ctas = tiles(BM, cand[i][0]) * cand[i][1];
       if (csk_ok(cand[i][0], cand[i][1]) && ctas <= sms && ctas * 10 >= static_cast<long long>(sms) * 7) {
@@ -520,7 +520,7 @@ int cg_set_tuning(cg_handle_t h, const cg_tuning_t* t) {
     return CG_OK;
   }
   if ((t->tile_n != 0 && t->tile_n != 64 && t->tile_n != 128 && t->tile_n != 256 && t->tile_n != 512) || t->cta_group < 0 ||
-      t->cta_group > 2 || t->cluster_split < 0 || t->cluster_split > 8 || t->num_units < 0 || t->dp_units < 0 || t->stages < 0 || t->group_m < 0 || t->max_ctas < 0)
+      t->cta_group > 2 || t->cluster_split < 0 || t->cluster_split > 4 || t->cluster_split == 3 || t->num_units < 0 || t->dp_units < 0 || t->stages < 0 || t->group_m < 0 || t->max_ctas < 0)
     return fail(h, CG_ERR_INVALID_ARG, "bad tuning values");
   h->tuning = *t;
   return CG_OK;

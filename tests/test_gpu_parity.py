@@ -114,6 +114,38 @@ def test_heuristic_splits_a_thin_last_wave(ctx, oracle):
     assert plan["dp_units"] == 12 and plan["num_units"] == 12
 
 
+@pytest.mark.parametrize("colmajor", [False, True])
+@pytest.mark.parametrize("tile_n,parts", [(128, 2), (256, 2), (256, 4)])
+def test_cluster_split_k(ctx, oracle, tile_n, parts, colmajor):
+    """K parts of a tile on the CTAs of one cluster, reduced through distributed shared memory."""
+    fl = W.FLAG_B_COLMAJOR if colmajor else 0
+    p = W.make(300, 1000, 1024, batch=2, seed=parts + tile_n, act=fl | W.ACT_RELU, alpha=2.0, beta=-1.0, A=SI, B=SI, bias=SI, R=SI)
+    plan = check(ctx, oracle, p, exact=True, tile_n=tile_n, cluster_split=parts)
+    assert plan["cluster_split"] == parts and plan["grid"] == plan["num_tiles"] * parts and plan["cta_group"] == 1
+    q = W.make(128, 512, 2048, seed=3, act=fl | W.ACT_SILU, A=("normal", 1.0), B=("normal", 0.03), bias=("normal", 1.0))
+    check(ctx, oracle, q, tile_n=tile_n, cluster_split=parts)
+    dev = PU.to_device(q)
+    first = PU.run_gpu(ctx, q, dev)
+    for _ in range(5):                                # parts are summed in part order: bitwise repeatable
+        assert np.array_equal(PU.run_gpu(ctx, q, dev), first)
+
+
+def test_cluster_split_is_chosen_for_skinny_problems_and_rejected_when_it_cannot_fit(ctx, oracle):
+    import paper_2604_01489_b200 as cg
+    p = W.make(128, 8192, 1024, seed=9, act=W.ACT_SILU | W.FLAG_B_COLMAJOR, A=("normal", 1.0), B=("normal", 0.03), bias=("normal", 1.0))
+    plan = check(ctx, oracle, p)
+    assert plan["cluster_split"] >= 2 and plan["cta_group"] == 1
+    dev = PU.to_device(p)
+    ctx.set_tuning(reset=True)
+    ctx.set_tuning(tile_n=128, cluster_split=4)       # 32 columns per CTA: below the 64-column minimum
+    assert cg.cg_gemm_epilogue(ctx.handle, dev["A"], dev["B"], dev["bias"], None, dev["D"], p.M, p.N, p.K, 1, 1.0, 0.0, p.act) == cg.CG_ERR_UNSUPPORTED
+    ctx.set_tuning(reset=True)
+    ctx.set_tuning(cluster_split=1)                   # 1 = never: falls back to the workspace split
+    PU.run_gpu(ctx, p, dev)
+    assert ctx.last_plan()["cluster_split"] == 1
+    ctx.set_tuning(reset=True)
+
+
 def test_stream_k_with_fewer_ctas_than_units_and_colmajor(ctx, oracle):
     p = W.make(200, 320, 1032, batch=2, seed=3, act=W.FLAG_B_COLMAJOR, A=SI, B=SI, alpha=1.0, beta=2.0, R=SI)
     check(ctx, oracle, p, exact=True, tile_n=64, cta_group=1, num_units=37, max_ctas=4)
