@@ -545,7 +545,8 @@ int cg_last_error(cg_handle_t h, int sync, char* buf, size_t len) {
     if (e != cudaSuccess) {
       code = fail(h, CG_ERR_CUDA, "device synchronisation failed: %s", cudaGetErrorString(e));
     } else if (dev != 0) {
-      code = fail(h, dev, "a bounded wait inside the kernel expired (device status %d)", dev);
+      code = fail(h, dev, dev == CG_ERR_TIMEOUT ? "a bounded wait inside the kernel expired (device status %d)"
+                                                : "the kernel's shared-memory layout did not fit (device status %d)", dev);
       // a timed-out split tile may have left tickets behind
       cudaMemset(h->tickets, 0, static_cast<size_t>(MAX_TICKET_TILES) * TICKETS_PER_TILE * sizeof(int));
     } else {
