@@ -2,7 +2,8 @@
 ad-hoc test problems.  Pure data: no arithmetic of the method lives here.
 
 Activation / flag encoding of the ``act`` argument (shared by the C ABI and the oracle's C ABI):
-low byte = activation (0 none, 1 ReLU, 2 GELU-tanh, 3 SiLU); bit 8 = B stored column-major
+low byte = activation (0 none, 1 ReLU, 2 GELU-tanh, 3 SiLU, 4 GELU-erf, 5 sigmoid, 6 tanh,
+7 leaky ReLU with slope 0.01); bit 8 = B stored column-major
 ([batch,N,K]); bit 9 = bias is bf16 instead of fp32.
 """
 from __future__ import annotations
@@ -16,6 +17,7 @@ import numpy as np
 from . import gen
 
 ACT_NONE, ACT_RELU, ACT_GELU_TANH, ACT_SILU = 0, 1, 2, 3
+ACT_GELU_ERF, ACT_SIGMOID, ACT_TANH, ACT_LEAKY_RELU = 4, 5, 6, 7
 FLAG_B_COLMAJOR = 1 << 8
 FLAG_BIAS_BF16 = 1 << 9
 

@@ -25,8 +25,9 @@
 // Readings where the paper is silent (all listed in the design notes):
 //   alpha scales A*B only; bias is a length-N vector broadcast over rows and batch and is not
 //   scaled; the activation comes before the residual; beta scales R only; when beta == 0, R
-//   is never read; GELU is the tanh form with constants sqrt(2/pi) and 0.044715; the bf16
-//   output is rounded to nearest-even directly from fp64.
+//   is never read; GELU is the tanh form with constants sqrt(2/pi) and 0.044715 (code 2) or the
+//   erf form (code 4); leaky ReLU has the fixed slope 0.01; the bf16 output is rounded to
+//   nearest-even directly from fp64.
 //
 // Pins (tests/test_oracle_*.py): identity and all-ones operands, small-integer operands
 // against an int64 contraction, a pure-Python triple loop on tiny shapes, numpy/torch fp64
@@ -71,7 +72,11 @@ inline uint16_t f64_to_bf16_rne(double v) {
   return sign | static_cast<uint16_t>(w >> 16);
 }
 
-enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU_TANH = 2, ACT_SILU = 3 };
+enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU_TANH = 2, ACT_SILU = 3,
+       // wider consumer family of the Level-2 prompt ("activation" among the consumers of a producer)
+       ACT_GELU_ERF = 4, ACT_SIGMOID = 5, ACT_TANH = 6, ACT_LEAKY_RELU = 7 };
+constexpr int ACT_LAST = ACT_LEAKY_RELU;
+constexpr double LEAKY_SLOPE = 0.01;
 enum { FLAG_B_COLMAJOR = 1 << 8, FLAG_BIAS_BF16 = 1 << 9 };
 
 inline double activation(int act, double t) {
@@ -82,6 +87,14 @@ inline double activation(int act, double t) {
       return t / (1.0 + std::exp(-t));
     case ACT_GELU_TANH:
       return 0.5 * t * (1.0 + std::tanh(0.7978845608028654 * (t + 0.044715 * t * t * t)));
+    case ACT_GELU_ERF:
+      return 0.5 * t * (1.0 + std::erf(t * 0.7071067811865476));
+    case ACT_SIGMOID:
+      return 1.0 / (1.0 + std::exp(-t));
+    case ACT_TANH:
+      return std::tanh(t);
+    case ACT_LEAKY_RELU:
+      return t > 0.0 ? t : LEAKY_SLOPE * t;
     default:
       return t;
   }
@@ -149,7 +162,7 @@ Problem make(const void* A, const void* B, const void* bias, const void* R, int6
 }
 
 bool bad(const Problem& p) {
-  return !p.A || !p.B || p.M < 1 || p.N < 1 || p.K < 1 || p.batch < 1 || p.act < 0 || p.act > 3 ||
+  return !p.A || !p.B || p.M < 1 || p.N < 1 || p.K < 1 || p.batch < 1 || p.act < 0 || p.act > ACT_LAST ||
          (p.beta != 0.0 && !p.R);
 }
 

@@ -16,6 +16,7 @@ import subprocess
 import numpy as np
 
 ACT_NONE, ACT_RELU, ACT_GELU_TANH, ACT_SILU = 0, 1, 2, 3
+ACT_GELU_ERF, ACT_SIGMOID, ACT_TANH, ACT_LEAKY_RELU = 4, 5, 6, 7
 FLAG_B_COLMAJOR = 1 << 8
 FLAG_BIAS_BF16 = 1 << 9
 

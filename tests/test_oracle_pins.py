@@ -116,7 +116,9 @@ def test_vs_numpy_fp64_matmul(oracle):
 def test_vs_torch_fp64_fused_reference(oracle):
     """Library special case: torch CPU float64 matmul + its own gelu(tanh)/silu/relu."""
     for act, fn in ((W.ACT_GELU_TANH, lambda t: torch.nn.functional.gelu(t, approximate="tanh")),
-                    (W.ACT_SILU, torch.nn.functional.silu), (W.ACT_RELU, torch.relu)):
+                    (W.ACT_SILU, torch.nn.functional.silu), (W.ACT_RELU, torch.relu),
+                    (W.ACT_GELU_ERF, torch.nn.functional.gelu), (W.ACT_SIGMOID, torch.sigmoid), (W.ACT_TANH, torch.tanh),
+                    (W.ACT_LEAKY_RELU, lambda t: torch.nn.functional.leaky_relu(t, 0.01))):
         p = W.make(33, 40, 64, 2, seed=21, act=act, alpha=1.25, beta=0.5, A=("normal", 1.0),
                    B=("normal", 0.2), bias=("normal", 1.0), R=("normal", 1.0))
         a, b, r = (torch.from_numpy(f64(x)) for x in (p.A, p.B, p.R))
@@ -219,7 +221,8 @@ def test_bf16_bias_flag(oracle):
 # ---------------------------------------------------------------- activations
 
 def test_activation_closed_forms(oracle):
-    kinds = {"silu": W.ACT_SILU, "gelu_tanh": W.ACT_GELU_TANH}
+    kinds = {"silu": W.ACT_SILU, "gelu_tanh": W.ACT_GELU_TANH, "gelu_erf": W.ACT_GELU_ERF, "sigmoid": W.ACT_SIGMOID,
+             "tanh": W.ACT_TANH, "leaky_relu": W.ACT_LEAKY_RELU}
     n = 0
     with open(os.path.join(GOLDEN, "activation_closed_forms.txt")) as f:
         for line in f:
@@ -229,7 +232,7 @@ def test_activation_closed_forms(oracle):
             got = oracle.activation(kinds[name], float(x))
             assert abs(got - float(want)) <= 1e-14 * abs(float(want)) + 1e-17, (name, x, got, want)
             n += 1
-    assert n == 22
+    assert n == 66
     assert oracle.activation(W.ACT_RELU, -1.0) == 0.0 and oracle.activation(W.ACT_RELU, 2.0) == 2.0
     assert oracle.activation(W.ACT_NONE, -3.25) == -3.25
 
@@ -244,6 +247,12 @@ def test_activation_identities(oracle):
         z = math.sqrt(2.0 / math.pi) * (x + 0.044715 * x ** 3)
         assert abs(oracle.activation(W.ACT_GELU_TANH, x) - x / (1.0 + math.exp(-2.0 * z))) < 1e-14 * max(1.0, abs(x))
         assert oracle.activation(W.ACT_RELU, x) == max(x, 0.0)
+        assert abs(oracle.activation(W.ACT_GELU_ERF, x) - oracle.activation(W.ACT_GELU_ERF, -x) - x) < 1e-14
+        assert abs(oracle.activation(W.ACT_SIGMOID, x) + oracle.activation(W.ACT_SIGMOID, -x) - 1.0) < 1e-15
+        assert oracle.activation(W.ACT_TANH, x) == -oracle.activation(W.ACT_TANH, -x)
+        assert abs(oracle.activation(W.ACT_SILU, x) - x * oracle.activation(W.ACT_SIGMOID, x)) < 1e-14 * max(1.0, abs(x))
+        assert abs(2.0 * oracle.activation(W.ACT_SIGMOID, 2.0 * x) - 1.0 - oracle.activation(W.ACT_TANH, x)) < 1e-14
+        assert oracle.activation(W.ACT_LEAKY_RELU, x) == (x if x > 0 else 0.01 * x)
 
 
 # ---------------------------------------------------------------- bf16 rounding
@@ -298,6 +307,6 @@ def test_output_bf16_is_rne_of_fp64_result(oracle):
 def test_rejects_bad_arguments(oracle):
     a = np.zeros((1, 8, 8), dtype=np.uint16)
     with pytest.raises(ValueError):
-        oracle.gemm_epilogue(a, a, None, None, 8, 8, 8, 1, 1.0, 0.0, 7)          # unknown activation
+        oracle.gemm_epilogue(a, a, None, None, 8, 8, 8, 1, 1.0, 0.0, 8)          # unknown activation
     with pytest.raises(ValueError):
         oracle.gemm_epilogue(a, a, None, None, 8, 8, 4, 1, 1.0, 0.0, 0)          # size mismatch
