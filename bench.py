@@ -294,6 +294,22 @@ def small_problem_extras(ctx, p, dev, flush):
     return {"us_graph_replay_per_launch": min(ts) * 1e6, "us_measurement_floor_one_element_fill": floor * 1e6}
 
 
+ACT_NAMES = {W.ACT_NONE: "none", W.ACT_RELU: "relu", W.ACT_GELU_TANH: "gelu_tanh", W.ACT_SILU: "silu",
+             W.ACT_GELU_ERF: "gelu_erf", W.ACT_SIGMOID: "sigmoid", W.ACT_TANH: "tanh", W.ACT_LEAKY_RELU: "leaky_relu"}
+
+
+def activation_sweep(ctx, p, dev, flush):
+    """The same problem under every activation code: what each epilogue costs on top of the main loop."""
+    import dataclasses
+    out = {}
+    for kind, label in ACT_NAMES.items():
+        q = dataclasses.replace(p, act=(p.act & ~0xFF) | kind)
+        per_launch_times(ctx, q, dev, 2, flush)
+        out[label] = min(per_launch_times(ctx, q, dev, 10, flush)) * 1e6
+    ctx.check()
+    return out
+
+
 def workload_table(ctx, device, peaks, names):
     """All five workloads under the heuristic plan, each launch timed alone after an L2 flush (their
     inputs may fit in L2)."""
@@ -318,6 +334,8 @@ def workload_table(ctx, device, peaks, names):
         if BOUND[name] == "latency":
             row.update(small_problem_extras(ctx, p, dev, flush))
         out[name] = row
+        if name == "cfg2_4096_gelu":
+            out["activation_sweep_4096_us_best"] = activation_sweep(ctx, p, dev, flush)
         del dev
     return out
 

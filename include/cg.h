@@ -49,7 +49,17 @@ enum {
 };
 
 /* Low byte of `act`. */
-enum { CG_ACT_NONE = 0, CG_ACT_RELU = 1, CG_ACT_GELU_TANH = 2, CG_ACT_SILU = 3 };
+enum {
+  CG_ACT_NONE = 0,
+  CG_ACT_RELU = 1,
+  CG_ACT_GELU_TANH = 2, /* t/2 * (1 + tanh(sqrt(2/pi) * (t + 0.044715 t^3))) */
+  CG_ACT_SILU = 3,      /* t / (1 + e^-t) */
+  /* further consumers of the same producer (the fusion rule's "activation" covers any pointwise map) */
+  CG_ACT_GELU_ERF = 4,  /* t/2 * (1 + erf(t / sqrt 2)) */
+  CG_ACT_SIGMOID = 5,   /* 1 / (1 + e^-t) */
+  CG_ACT_TANH = 6,
+  CG_ACT_LEAKY_RELU = 7 /* t > 0 ? t : 0.01 t  (fixed slope) */
+};
 /* OR-ed into `act`: operand layout / dtype that the argument list has no slot for. */
 enum {
   CG_FLAG_B_COLMAJOR = 1 << 8, /* B is stored [batch,N,K] (element (k,n) at n*K + k) */

@@ -14,6 +14,7 @@ from . import build as _build
 
 CG_OK, CG_ERR_INVALID_ARG, CG_ERR_UNSUPPORTED, CG_ERR_ARCH, CG_ERR_CUDA, CG_ERR_WORKSPACE, CG_ERR_TIMEOUT = range(7)
 CG_ACT_NONE, CG_ACT_RELU, CG_ACT_GELU_TANH, CG_ACT_SILU = 0, 1, 2, 3
+CG_ACT_GELU_ERF, CG_ACT_SIGMOID, CG_ACT_TANH, CG_ACT_LEAKY_RELU = 4, 5, 6, 7
 CG_FLAG_B_COLMAJOR = 1 << 8
 CG_FLAG_BIAS_BF16 = 1 << 9
 

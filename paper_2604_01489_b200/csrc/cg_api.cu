@@ -325,7 +325,7 @@ int validate(cg_context* h, const void* A, const void* B, const void* bias, cons
   if (!A || !B || !D) return fail(h, CG_ERR_INVALID_ARG, "A, B and D must not be NULL");
   if (M < 1 || N < 1 || K < 1 || batch < 1) return fail(h, CG_ERR_INVALID_ARG, "M, N, K, batch must be >= 1");
   const int kind = act & 0xFF;
-  if (kind > CG_ACT_SILU || (act & ~(0xFF | CG_FLAG_B_COLMAJOR | CG_FLAG_BIAS_BF16)) != 0 || act < 0)
+  if (kind > CG_ACT_LEAKY_RELU || (act & ~(0xFF | CG_FLAG_B_COLMAJOR | CG_FLAG_BIAS_BF16)) != 0 || act < 0)
     return fail(h, CG_ERR_INVALID_ARG, "unknown activation or flag bits in act=0x%x", act);
   if (beta != 0.0f && !R) return fail(h, CG_ERR_INVALID_ARG, "R must not be NULL when beta != 0");
   if (N % 8 != 0 || K % 8 != 0) return fail(h, CG_ERR_UNSUPPORTED, "N and K must be multiples of 8 (got N=%d K=%d)", N, K);

@@ -60,7 +60,8 @@ constexpr int EPI_COLS = 64;        // columns per epilogue chunk (one 128-byte 
 constexpr int EPI_BUF_BYTES = 32 * EPI_COLS * 2;   // one warp's staging buffer: 32 rows x 128 B
 constexpr int CTRL_BYTES = 256;
 
-enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU_TANH = 2, ACT_SILU = 3 };
+enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU_TANH = 2, ACT_SILU = 3,
+       ACT_GELU_ERF = 4, ACT_SIGMOID = 5, ACT_TANH = 6, ACT_LEAKY_RELU = 7 };
 enum { STATUS_OK = 0, STATUS_SMEM = 4, STATUS_TIMEOUT = 6 };
 
 struct KernelParams {
@@ -228,6 +229,14 @@ __device__ __forceinline__ float activate(float t) {
     // 0.5 t (1 + tanh z) = t * sigmoid(2 z),  z = sqrt(2/pi) (t + 0.044715 t^3)
     const float z2 = 1.5957691216057308f * (t + 0.044715f * t * t * t);
     return __fdividef(t, 1.0f + __expf(-z2));
+  } else if constexpr (ACT == ACT_GELU_ERF) {
+    return 0.5f * t * (1.0f + erff(0.70710678118654752f * t));
+  } else if constexpr (ACT == ACT_SIGMOID) {
+    return __fdividef(1.0f, 1.0f + __expf(-t));
+  } else if constexpr (ACT == ACT_TANH) {
+    return tanhf(t);
+  } else if constexpr (ACT == ACT_LEAKY_RELU) {
+    return t > 0.0f ? t : 0.01f * t;
   } else {
     return t;
   }
@@ -755,24 +764,25 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           bias_s[lane + 32] = bv1;
           __syncwarp();
           uint32_t outw[EPI_COLS / 2];
+#define CG_EPILOGUE_CASE(ACT)                                                              \
+  case ACT:                                                                                \
+    if (has_r) epilogue_chunk<ACT, true>(accv, bias_s, p.alpha, p.beta, rq, outw);         \
+    else epilogue_chunk<ACT, false>(accv, bias_s, p.alpha, p.beta, rq, outw);              \
+    break;
           switch (p.act) {
-            case ACT_RELU:
-              if (has_r) epilogue_chunk<ACT_RELU, true>(accv, bias_s, p.alpha, p.beta, rq, outw);
-              else epilogue_chunk<ACT_RELU, false>(accv, bias_s, p.alpha, p.beta, rq, outw);
-              break;
-            case ACT_GELU_TANH:
-              if (has_r) epilogue_chunk<ACT_GELU_TANH, true>(accv, bias_s, p.alpha, p.beta, rq, outw);
-              else epilogue_chunk<ACT_GELU_TANH, false>(accv, bias_s, p.alpha, p.beta, rq, outw);
-              break;
-            case ACT_SILU:
-              if (has_r) epilogue_chunk<ACT_SILU, true>(accv, bias_s, p.alpha, p.beta, rq, outw);
-              else epilogue_chunk<ACT_SILU, false>(accv, bias_s, p.alpha, p.beta, rq, outw);
-              break;
+            CG_EPILOGUE_CASE(ACT_RELU)
+            CG_EPILOGUE_CASE(ACT_GELU_TANH)
+            CG_EPILOGUE_CASE(ACT_SILU)
+            CG_EPILOGUE_CASE(ACT_GELU_ERF)
+            CG_EPILOGUE_CASE(ACT_SIGMOID)
+            CG_EPILOGUE_CASE(ACT_TANH)
+            CG_EPILOGUE_CASE(ACT_LEAKY_RELU)
             default:
               if (has_r) epilogue_chunk<ACT_NONE, true>(accv, bias_s, p.alpha, p.beta, rq, outw);
               else epilogue_chunk<ACT_NONE, false>(accv, bias_s, p.alpha, p.beta, rq, outw);
               break;
           }
+#undef CG_EPILOGUE_CASE
           // staging buffer free again?  (the store that last used it has finished reading it) --
           // asked only now, after the arithmetic, so that the wait overlaps it
           if (lane == 0) ptx::bulk_wait_group_read<C::EPI_BUFS - 1>();

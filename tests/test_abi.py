@@ -43,6 +43,7 @@ def test_constants_match_header():
     from paper_2604_01489_b200 import binding
     for name in ("CG_OK", "CG_ERR_INVALID_ARG", "CG_ERR_UNSUPPORTED", "CG_ERR_ARCH", "CG_ERR_CUDA", "CG_ERR_WORKSPACE",
                  "CG_ERR_TIMEOUT", "CG_ACT_NONE", "CG_ACT_RELU", "CG_ACT_GELU_TANH", "CG_ACT_SILU",
+                 "CG_ACT_GELU_ERF", "CG_ACT_SIGMOID", "CG_ACT_TANH", "CG_ACT_LEAKY_RELU",
                  "CG_FLAG_B_COLMAJOR", "CG_FLAG_BIAS_BF16"):
         assert getattr(binding, name) == header_enum(name), name
     from cg_inputs import workloads as W
@@ -51,6 +52,8 @@ def test_constants_match_header():
         assert mod.ACT_RELU == binding.CG_ACT_RELU and mod.ACT_GELU_TANH == binding.CG_ACT_GELU_TANH
         assert mod.ACT_SILU == binding.CG_ACT_SILU and mod.FLAG_B_COLMAJOR == binding.CG_FLAG_B_COLMAJOR
         assert mod.FLAG_BIAS_BF16 == binding.CG_FLAG_BIAS_BF16
+        assert (mod.ACT_GELU_ERF, mod.ACT_SIGMOID, mod.ACT_TANH, mod.ACT_LEAKY_RELU) == (
+            binding.CG_ACT_GELU_ERF, binding.CG_ACT_SIGMOID, binding.CG_ACT_TANH, binding.CG_ACT_LEAKY_RELU)
 
 
 def test_struct_layouts_match_header():

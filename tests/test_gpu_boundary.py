@@ -48,7 +48,7 @@ def test_error_codes_and_D_untouched(cg, ctx):
     assert call(D=None) == cg.CG_ERR_INVALID_ARG
     assert call(M=0) == cg.CG_ERR_INVALID_ARG and call(N=-8) == cg.CG_ERR_INVALID_ARG
     assert call(K=0) == cg.CG_ERR_INVALID_ARG and call(batch=0) == cg.CG_ERR_INVALID_ARG
-    assert call(act=4) == cg.CG_ERR_INVALID_ARG and call(act=1 << 12) == cg.CG_ERR_INVALID_ARG
+    assert call(act=8) == cg.CG_ERR_INVALID_ARG and call(act=1 << 12) == cg.CG_ERR_INVALID_ARG
     assert call(beta=1.0) == cg.CG_ERR_INVALID_ARG                      # R missing
     assert call(N=60) == cg.CG_ERR_UNSUPPORTED and call(K=36) == cg.CG_ERR_UNSUPPORTED
     assert call(A=A.data_ptr() + 2) == cg.CG_ERR_UNSUPPORTED            # misaligned operand

@@ -165,7 +165,10 @@ def test_split_k_random_inputs_and_determinism(ctx, oracle):
 
 # ------------------------------------------------------------------ epilogue variants, random inputs
 
-@pytest.mark.parametrize("act", [W.ACT_NONE, W.ACT_RELU, W.ACT_GELU_TANH, W.ACT_SILU])
+ALL_ACTS = [W.ACT_NONE, W.ACT_RELU, W.ACT_GELU_TANH, W.ACT_SILU, W.ACT_GELU_ERF, W.ACT_SIGMOID, W.ACT_TANH, W.ACT_LEAKY_RELU]
+
+
+@pytest.mark.parametrize("act", ALL_ACTS)
 @pytest.mark.parametrize("bias", [None, "f32", "bf16"])
 @pytest.mark.parametrize("residual", [False, True])
 def test_epilogue_variants(ctx, oracle, act, bias, residual):
@@ -179,10 +182,30 @@ def test_epilogue_variants(ctx, oracle, act, bias, residual):
 
 
 def test_activation_tails(ctx, oracle):
-    """Large |t| through SiLU / GELU: no NaN from exp overflow, correct limits."""
-    for act in (W.ACT_SILU, W.ACT_GELU_TANH):
+    """Large |t| through the exponential-based activations: no NaN from exp overflow, correct limits."""
+    for act in (W.ACT_SILU, W.ACT_GELU_TANH, W.ACT_GELU_ERF, W.ACT_SIGMOID, W.ACT_TANH):
         p = W.make(128, 64, 64, seed=1, act=act, alpha=40.0, A=("uniform", 1.0), B=("uniform", 1.0), bias=("normal", 30.0))
         check(ctx, oracle, p)
+
+
+@pytest.mark.parametrize("act", ALL_ACTS[1:])
+def test_activation_curve_elementwise(ctx, oracle, act):
+    """K = 64 with A = identity block: the accumulator equals B exactly, so the output is the activation of
+    bf16 grid points spread over [-12, 12] and tightly around 0 -- compared at a far tighter bound than the
+    GEMM tolerance (2 bf16 ulps of the result plus 1e-6 absolute)."""
+    M = N = 128
+    K = 64
+    a = np.zeros((1, M, K), dtype=np.float32)
+    a[0, np.arange(M), np.arange(M) % K] = 1.0
+    g = np.random.default_rng(act)
+    vals = np.concatenate([g.uniform(-12, 12, K * N // 2), g.normal(0, 0.05, K * N // 2)]).astype(np.float32)
+    b = gen.bf16_bits_to_f32(gen.f32_to_bf16_bits(vals)).reshape(1, K, N)
+    p = W.make(M, N, K, seed=0, act=act)
+    p.A = gen.f32_to_bf16_bits(a)
+    p.B = gen.f32_to_bf16_bits(b)
+    d = gen.bf16_bits_to_f32(PU.run_gpu(ctx, p)).astype(np.float64)
+    d64, _ = oracle.gemm_epilogue(p.A, p.B, None, None, M, N, K, 1, 1.0, 0.0, act)
+    assert np.all(np.abs(d - d64) <= 2.0 ** -7 * np.abs(d64) + 1e-6)
 
 
 def test_beta_zero_ignores_R_and_alpha_zero_keeps_bias(ctx, oracle):
