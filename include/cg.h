@@ -124,6 +124,20 @@ typedef struct cg_tuning {
 } cg_tuning_t;
 CG_API int cg_set_tuning(cg_handle_t h, const cg_tuning_t* t /* NULL = reset */);
 
+/*
+ * Debug timeline (the profiling-summary idea of the paper's "Profiling-Driven Refinement" stage,
+ * taken inside the kernel).  With a non-NULL `device_buf` of at least max_ctas * 32 * 8 bytes
+ * (caller-owned device memory, 8-byte aligned), the first `max_ctas` CTAs of every following launch
+ * on this handle record global-timer nanoseconds of events into slots [cta * 32 + event]:
+ * 0 kernel entry, 1 set-up done, 2 first / 3 last operand load issued, 4 first operands landed,
+ * 5 last MMA issued, 6 last accumulator seen by the epilogue, 7 / 8 split-K exchange entered / left,
+ * 9 / 10 first / last output store of the last tile issued, 11 stores complete, 12 tensor memory
+ * freed, 13 / 14 / 15 first chunk of the last tile in registers / computed / staged; slots 16 and 17
+ * hold the SM's cycle counter at events 0 and 12 (their difference over the nanoseconds gives the
+ * SM clock during the launch).  A slot an event never reached keeps its old contents.  NULL or max_ctas == 0 turns it off.
+ */
+CG_API int cg_set_trace(cg_handle_t h, void* device_buf, int max_ctas);
+
 /* What the last successful cg_gemm_epilogue on this handle launched. */
 typedef struct cg_plan_info {
   int tile_m, tile_n, cta_group, stages, group_m;

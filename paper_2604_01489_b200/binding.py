@@ -21,7 +21,7 @@ CG_FLAG_BIAS_BF16 = 1 << 9
 STATUS_NAMES = {0: "CG_OK", 1: "CG_ERR_INVALID_ARG", 2: "CG_ERR_UNSUPPORTED", 3: "CG_ERR_ARCH", 4: "CG_ERR_CUDA",
                 5: "CG_ERR_WORKSPACE", 6: "CG_ERR_TIMEOUT"}
 
-EXPORTS = ["cg_create", "cg_gemm_epilogue", "cg_gemm_epilogue_host", "cg_set_tuning", "cg_get_last_plan",
+EXPORTS = ["cg_create", "cg_gemm_epilogue", "cg_gemm_epilogue_host", "cg_set_tuning", "cg_set_trace", "cg_get_last_plan",
            "cg_last_error", "cg_gemm_epilogue_noalloc", "cg_destroy"]
 
 
@@ -66,6 +66,7 @@ def load() -> ctypes.CDLL:
     lib.cg_gemm_epilogue.argtypes = gemm_args
     lib.cg_gemm_epilogue_host.argtypes = gemm_args
     lib.cg_set_tuning.argtypes = [vp, ctypes.POINTER(cg_tuning_t)]
+    lib.cg_set_trace.argtypes = [vp, vp, ci]
     lib.cg_get_last_plan.argtypes = [vp, ctypes.POINTER(cg_plan_info_t)]
     lib.cg_last_error.argtypes = [vp, ci, ctypes.c_char_p, sz]
     lib.cg_destroy.argtypes = [vp]
@@ -145,6 +146,11 @@ def cg_set_tuning(h, tile_n=0, cta_group=0, num_units=0, dp_units=0, stages=0, g
     return load().cg_set_tuning(h, ctypes.byref(t))
 
 
+def cg_set_trace(h, device_buf, max_ctas: int) -> int:
+    """device_buf: int64 CUDA tensor of at least max_ctas * 32 elements (or None to switch tracing off)."""
+    return load().cg_set_trace(h, _dev_ptr(device_buf), int(max_ctas))
+
+
 def cg_get_last_plan(h) -> dict:
     info = cg_plan_info_t()
     rc = load().cg_get_last_plan(h, ctypes.byref(info))
@@ -194,6 +200,11 @@ class Context:
         rc = cg_set_tuning(self.handle, **kw)
         if rc != CG_OK:
             raise CgError(rc, cg_last_error(self.handle)[1])
+
+    def set_trace(self, device_buf, max_ctas: int):
+        rc = cg_set_trace(self.handle, device_buf, max_ctas)
+        if rc != CG_OK:
+            raise CgError(rc, "cg_set_trace failed")
 
     def last_plan(self) -> dict:
         return cg_get_last_plan(self.handle)

@@ -29,7 +29,7 @@ constexpr int TICKETS_PER_TILE = 8;                // one ticket per epilogue wa
 
 struct Plan {
   int bn, cg, stages, group_m, num_units, dp_units, grid, num_workers, cluster_split;
-  int tiles_m, tiles_n, num_tiles, k_blocks, smem;
+  int tiles_m, tiles_n, num_tiles, k_blocks, smem, r_shared;
   bool b_kmajor;
 };
 
@@ -75,6 +75,10 @@ struct cg_context {
   long long wait_limit = 4000000000ll;   // about two seconds of SM clocks
   int test_starve = 0;                   // test hook (CG_TEST_STARVE): see KernelParams::test_starve
   bool log_plans = false;                // CG_LOG
+  int r_shared = -1;                     // CG_R_SHARED: 0 / 1 force the residual's buffer choice (ablation), else heuristic
+  int split_first = 1;                   // CG_SPLIT_FIRST=0 restores the old order (ablation)
+  unsigned long long* trace = nullptr;   // cg_set_trace
+  int trace_ctas = 0;
   MapCacheEntry map_cache[MAP_CACHE_SIZE];
   int map_cache_next = 0;
   StagingBuf sA, sB, sBias, sR, sD;
@@ -302,14 +306,19 @@ int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, bool
   pl->grid = pl->num_workers * cgn;
   pl->cluster_split = csk;
 
-  const int smax = has_r ? e.stages_max_r : e.stages_max;       // the residual's chunk buffers cost ring depth
+  // The residual chunks either get buffers of their own (requested a chunk ahead of their use) or
+  // land in the output staging buffers (requested after the previous store has read them): the
+  // second form frees shared memory, and is taken when that buys the ring another stage.
+  pl->r_shared = (has_r && (h->r_shared >= 0 ? h->r_shared != 0 : e.stages_max > e.stages_max_r)) ? 1 : 0;
+  const bool r_own = has_r && !pl->r_shared;
+  const int smax = r_own ? e.stages_max_r : e.stages_max;       // the residual's chunk buffers cost ring depth
   int stages = t.stages > 0 ? t.stages : smax;
   if (stages > smax) stages = smax;
   if (stages < 1) stages = 1;
   if (csk > 1 && static_cast<long long>(stages) * e.stage_bytes < static_cast<long long>(BM) * bn * 4)
     return fail(h, CG_ERR_UNSUPPORTED, "cluster split needs a ring of at least %d bytes for the partial tiles", BM * bn * 4);
   pl->stages = stages;
-  pl->smem = stages * e.stage_bytes + e.fixed_bytes + (has_r ? e.r_bytes : 0) + 1024;   // layout + alignment slack, capped
+  pl->smem = stages * e.stage_bytes + e.fixed_bytes + (r_own ? e.r_bytes : 0) + 1024;   // layout + alignment slack, capped
   if (pl->smem > SMEM_LIMIT) pl->smem = SMEM_LIMIT;
 
   int gm = t.group_m > 0 ? t.group_m : (bn == 512 ? 16 : 8);
@@ -373,6 +382,10 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   p.num_workers = pl.num_workers;
   p.stages = pl.stages;
   p.cluster_split = pl.cluster_split;
+  p.r_shared = pl.r_shared;
+  p.split_first = (h->split_first && pl.cluster_split <= 1 && pl.dp_units > 0 && pl.dp_units < pl.num_units) ? 1 : 0;
+  p.trace = h->trace;
+  p.trace_ctas = h->trace_ctas;
   p.alpha = alpha; p.beta = beta;
   p.act = act & 0xFF;
   p.bias_bf16 = (act & CG_FLAG_BIAS_BF16) ? 1 : 0;
@@ -471,6 +484,8 @@ int cg_create(cg_handle_t* out, int device, size_t workspace_bytes) {
   }
   if (const char* w = getenv("CG_TEST_STARVE")) h->test_starve = atoi(w) != 0;
   h->log_plans = getenv("CG_LOG") != nullptr;
+  if (const char* w = getenv("CG_R_SHARED")) h->r_shared = atoi(w);
+  if (const char* w = getenv("CG_SPLIT_FIRST")) h->split_first = atoi(w);
   *out = h;
   return CG_OK;
 }
@@ -523,6 +538,14 @@ int cg_set_tuning(cg_handle_t h, const cg_tuning_t* t) {
       t->cta_group > 2 || t->cluster_split < 0 || t->cluster_split > 4 || t->cluster_split == 3 || t->num_units < 0 || t->dp_units < 0 || t->stages < 0 || t->group_m < 0 || t->max_ctas < 0)
     return fail(h, CG_ERR_INVALID_ARG, "bad tuning values");
   h->tuning = *t;
+  return CG_OK;
+}
+
+int cg_set_trace(cg_handle_t h, void* device_buf, int max_ctas) {
+  if (!h || max_ctas < 0 || (device_buf && (reinterpret_cast<uintptr_t>(device_buf) & 7) != 0)) return CG_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(h->mu);
+  h->trace = (device_buf && max_ctas > 0) ? static_cast<unsigned long long*>(device_buf) : nullptr;
+  h->trace_ctas = h->trace ? max_ctas : 0;
   return CG_OK;
 }
 

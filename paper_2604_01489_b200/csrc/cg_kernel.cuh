@@ -74,8 +74,12 @@ struct KernelParams {
   int dp_units;           // the first dp_units units are whole tiles (unit u = tile u) ...
   int unit_q, unit_r;     // ... the rest cut the remaining iterations evenly: start = base + v*q + min(v, r)
   int num_workers;        // CTAs (CG == 1) or CTA pairs (CG == 2)
+  int split_first;        // workers take their units from the highest index down: the split units (which come
+                          // after the whole tiles in the numbering) run first, so that parking and reducing
+                          // partial tiles overlaps the main loops of the whole tiles instead of ending the launch
   int stages;
   int cluster_split;      // > 1: the CTAs of a cluster of this size hold the K parts of one tile (CG == 1 only)
+  int r_shared;           // the residual chunk lands in the output staging buffer itself (no buffers of its own)
   float alpha, beta;
   int act;
   int bias_bf16;
@@ -85,6 +89,8 @@ struct KernelParams {
   int* tickets;           // [num_tiles * CG * 8] (one per epilogue warp slot), zero between launches
   int* status;
   long long wait_limit;   // clock cycles before a wait gives up
+  unsigned long long* trace;   // debug: 32 slots of timestamps (globaltimer, ns) per CTA for the first trace_ctas CTAs, or NULL
+  int trace_ctas;
   int test_starve;        // test hook: the producer withholds the first A load, so `full[0]` never completes
 };
 
@@ -113,7 +119,7 @@ struct Cfg {
   static constexpr int R_BYTES = EPI_WARPS * EPI_BUF_BYTES;      // per warp: one 64-column chunk of the residual
   static constexpr int FIXED_BYTES = EPI_BYTES + BIAS_BYTES + CTRL_BYTES;   // + R_BYTES when there is a residual
   // Up to 1023 bytes go to aligning the ring; the kernel checks that what is left suffices.
-  __host__ __device__ static constexpr int stages_max(bool with_r) {
+  __host__ __device__ static constexpr int stages_max(bool with_r) {   // with_r: residual buffers of their own
     const int fit = (SMEM_LIMIT - FIXED_BYTES - (with_r ? R_BYTES : 0)) / STAGE_BYTES;
     return fit < MAX_STAGES ? fit : MAX_STAGES;
   }
@@ -159,13 +165,18 @@ struct Segment {
 // The sequence of (tile, k-range) segments a worker processes; all roles walk the same one.
 struct WorkIter {
   const KernelParams& p;
-  int unit, it, end;
+  int unit, step, it, end;
   bool head;
-  __device__ WorkIter(const KernelParams& p_, int worker) : p(p_), unit(worker - p_.num_workers), it(0), end(0), head(false) {}
+  __device__ WorkIter(const KernelParams& p_, int worker) : p(p_), unit(worker - p_.num_workers), step(p_.num_workers), it(0), end(0), head(false) {
+    if (p.split_first && worker < p.num_units) {
+      unit = worker + ((p.num_units - 1 - worker) / p.num_workers + 1) * p.num_workers;   // one step above this worker's last unit
+      step = -p.num_workers;
+    }
+  }
   __device__ bool next(Segment& s) {
     while (it >= end) {
-      unit += p.num_workers;
-      if (unit >= p.num_units) return false;
+      unit += step;
+      if (unit >= p.num_units || unit < 0) return false;
       it = unit_start(p, unit);
       end = unit_start(p, unit + 1);
       head = true;
@@ -198,6 +209,18 @@ __device__ __forceinline__ void decode_tile(const KernelParams& p, int tile, int
   const int rr = r - g * gsz;
   nt = rr / gm;
   mt = first_m + (rr - nt * gm);
+}
+
+// Debug timeline: event `ev` of this CTA, in nanoseconds of the global timer.
+enum { TR_START = 0, TR_SETUP_DONE, TR_FIRST_LOAD, TR_LAST_LOAD, TR_FIRST_FULL, TR_LAST_MMA, TR_ACC_SEEN, TR_EXCH_A,
+       TR_EXCH_B, TR_FIRST_STORE, TR_LAST_STORE, TR_STORES_DONE, TR_END, TR_EPI_LOADED, TR_EPI_MATH, TR_EPI_STAGED, TR_CLOCK_START, TR_CLOCK_END, TR_SLOTS = 32 };
+__device__ __forceinline__ void trace_event(const KernelParams& p, int ev) {
+  if (p.trace != nullptr && static_cast<int>(blockIdx.x) < p.trace_ctas) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    p.trace[blockIdx.x * TR_SLOTS + ev] = t;
+    if (ev == TR_START || ev == TR_END) p.trace[blockIdx.x * TR_SLOTS + (ev == TR_START ? TR_CLOCK_START : TR_CLOCK_END)] = clock64();
+  }
 }
 
 // Bounded mbarrier wait.  false: gave up (limit expired here, or another role aborted).
@@ -301,14 +324,15 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   uint8_t* epi_ptr = smem + stages * C::STAGE_BYTES;
   const uint32_t epi_addr = ring_addr + stages * C::STAGE_BYTES;
   const bool has_r = (p.beta != 0.0f);
-  const int r_bytes = has_r ? C::R_BYTES : 0;           // residual chunks sit between the staging buffers and the bias
+  const bool r_shared = has_r && p.r_shared != 0;
+  const int r_bytes = (has_r && !r_shared) ? C::R_BYTES : 0;   // residual chunks sit between the staging buffers and the bias
   const uint32_t rbuf_addr = epi_addr + C::EPI_BYTES;
   float* bias_all = reinterpret_cast<float*>(epi_ptr + C::EPI_BYTES + r_bytes);
   Ctrl* ctrl = reinterpret_cast<Ctrl*>(epi_ptr + C::EPI_BYTES + r_bytes + C::BIAS_BYTES);
   {
     uint32_t dyn_bytes;
     asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn_bytes));
-    if (pad + static_cast<uint32_t>(C::layout_bytes(stages, has_r)) > dyn_bytes) {   // never expected: the ring would not fit
+    if (pad + static_cast<uint32_t>(C::layout_bytes(stages, has_r && !r_shared)) > dyn_bytes) {   // never expected: the ring would not fit
       if (threadIdx.x == 0) atomicCAS(p.status, STATUS_OK, STATUS_SMEM);
       return;
     }
@@ -321,6 +345,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 
   // ---- set-up: barriers, tensor memory
   if (threadIdx.x == 0) {
+    trace_event(p, TR_START);
     for (int s = 0; s < stages; ++s) {
       ptx::mbar_init(ptx::smem_u32(&ctrl->full[s]), 1);
       ptx::mbar_init(ptx::smem_u32(&ctrl->empty[s]), 1);
@@ -350,6 +375,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   }
   ptx::tc_fence_after();
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&ctrl->tmem_base);
+  if (threadIdx.x == 0) trace_event(p, TR_SETUP_DONE);
 
   if (warp == 0) {
     // ================================================================ producer
@@ -407,10 +433,12 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
               }
             }
           }
+          if (issued == 0) trace_event(p, TR_FIRST_LOAD);
           ++issued;
           if (++stage == stages) { stage = 0; phase ^= 1u; }
         }
       }
+      trace_event(p, TR_LAST_LOAD);
       if (!ok || *reinterpret_cast<volatile int*>(&ctrl->abort)) {
         // abort path: let the copies still in flight land before shared memory is given up.
         // The leader can watch its `full` barriers; either CTA also sits out a fixed settle
@@ -471,6 +499,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         uint32_t accumulate = 0;
         for (int kb = s.kb0; kb < s.kb1; ++kb) {
           if (!wait_bar(full0 + stage * 8, phase, ctrl, p)) { ok = false; break; }
+          if (accumulate == 0 && acc == 0 && acc_phase == 0) trace_event(p, TR_FIRST_FULL);
           ptx::tc_fence_after();
           const uint32_t a_lo = a_lo0 + stage * STAGE_STEP;
           const uint32_t b_lo = b_lo0 + stage * STAGE_STEP;
@@ -499,6 +528,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         if constexpr (CG == 2) ptx::tc_commit<CG>(ptx::mapa(full_local, 1));
         if (++acc == C::ACC_BUFS) { acc = 0; acc_phase ^= 1u; }
       }
+      trace_event(p, TR_LAST_MMA);
       if (!ok || *reinterpret_cast<volatile int*>(&ctrl->abort)) {
         // abort path: wait (bounded) until the MMAs issued so far have retired
         ptx::tc_commit<CG>(ptx::smem_u32(&ctrl->drain));
@@ -534,16 +564,37 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     // The residual reaches the epilogue through TMA: one 64-column chunk (32 rows x 128 B, same box
     // and swizzle as the output staging) per warp, requested one chunk -- and across tiles one
     // tile -- ahead of its use, so that the reads are coalesced and off the critical path.
+    // With `r_shared` the chunk lands in the staging buffer its output will leave from (each thread
+    // reads and later rewrites only its own row): no buffers of its own, so the ring keeps a stage
+    // more, but a request has to wait until the store that last used the buffer has read it, so it
+    // follows the chunk's store instead of preceding its arithmetic.
     const uint32_t rbuf = rbuf_addr + ew * EPI_BUF_BYTES;
     const uint32_t r_bar = ptx::smem_u32(&ctrl->r_full[ew]);
     uint32_t r_phase = 0;
     bool r_pending = false;          // a chunk has been requested and not yet read
-    auto request_residual = [&](int col, int row0, int bb) {
+    auto request_residual = [&](int col, int row0, int bb) {   // for the chunk that will be staged in `store_buf`
       if (lane == 0) {
+        uint32_t dst = rbuf;
+        if (r_shared) {
+          ptx::bulk_wait_group_read<0>();                       // every earlier store has read its buffer
+          dst = stage_base + store_buf * EPI_BUF_BYTES;
+        }
         ptx::mbar_arrive_expect_tx(r_bar, EPI_BUF_BYTES);
-        ptx::tma_load_3d(rbuf, &tmR, r_bar, col, row0, bb);     // outside the tensor: zero fill, same byte count
+        ptx::tma_load_3d(dst, &tmR, r_bar, col, row0, bb);      // outside the tensor: zero fill, same byte count
       }
       r_pending = true;
+    };
+    auto request_next_residual = [&](int c, int c_step, int c_hi, int n0, int row0, int bb, bool have_next,
+                                     const Segment& s_next, int c_lo) {
+      if (c + c_step < c_hi) {
+        request_residual(n0 + c_step * EPI_COLS, row0, bb);
+      } else if (have_next && s_next.kb0 == 0 && s_next.kb1 == p.k_blocks) {
+        // first chunk of the next whole tile, a main loop ahead
+        int nb2, nmt, nnt;
+        decode_tile(p, s_next.tile, nb2, nmt, nnt);
+        if (nnt * BN + c_lo * EPI_COLS < p.N)
+          request_residual(nnt * BN + c_lo * EPI_COLS, nmt * (BM * CG) + static_cast<int>(cta_rank) * BM + q * 32, nb2);
+      }
     };
     // Pulls this thread's row of a tile's residual (its share of the columns) into L2.
     auto prefetch_residual = [&](const Segment& sg) {
@@ -613,6 +664,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         bias_reg[2 * j + 1] = b1;
       }
       if (!wait_bar(ptx::smem_u32(&ctrl->acc_full[acc]), acc_phase, ctrl, p)) { ok = false; break; }
+      if (ew == 0 && lane == 0) trace_event(p, TR_ACC_SEEN);
       ptx::tc_fence_after();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(acc * BN);
       const uint32_t acc_empty_bar = (CG == 2) ? ptx::mapa(ptx::smem_u32(&ctrl->acc_empty[acc]), 0)
@@ -625,6 +677,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         ptx::cluster_arrive();                 // A: every CTA of the cluster is done with its operand ring
         ptx::cluster_wait();
         ++cluster_barriers_done;
+        if (ew == 0 && lane == 0) trace_event(p, TR_EXCH_A);
         constexpr int GROUPS32 = BN / 32 / C::EPI_COL_GROUPS;
         for (int c = col_group * GROUPS32; c < (col_group + 1) * GROUPS32; ++c) {
           uint32_t v[32];
@@ -646,6 +699,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         ptx::cluster_arrive();                 // B: all partial tiles have been delivered
         ptx::cluster_wait();
         ++cluster_barriers_done;
+        if (ew == 0 && lane == 0) trace_event(p, TR_EXCH_B);
       } else if (!whole_tile) {
         // ---- split tile: park the fp32 partial, draw a ticket
         const int slot = (2 * (s.unit - p.dp_units) + (s.head ? 0 : 1)) * CG + static_cast<int>(cta_rank);
@@ -683,6 +737,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         first_unit = __shfl_sync(0xFFFFFFFFu, first_unit, 0);
         last_unit = __shfl_sync(0xFFFFFFFFu, last_unit, 0);
         reduce = (last != 0);
+        if (ew == 0 && lane == 0) trace_event(p, TR_EXCH_B);
         if (reduce) {
           __threadfence();
           if (has_r && c_lo < c_hi) request_residual(n_base + c_lo * EPI_COLS, m_base + q * 32, b);
@@ -737,28 +792,22 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
               }
             }
           }
+          if (ew == 0 && lane == 0 && c == c_lo) trace_event(p, TR_EPI_LOADED);
           // residual of this chunk: this thread's row of the TMA-filled buffer (swizzled like the staging)
           uint4 rq[EPI_COLS / 8];
           if (has_r) {
             if (!wait_bar(r_bar, r_phase, ctrl, p)) { ok = false; break; }
             r_phase ^= 1u;
             r_pending = false;
+            const uint32_t rsrc = r_shared ? stage_base + store_buf * EPI_BUF_BYTES : rbuf;
 #pragma unroll
             for (int j = 0; j < EPI_COLS / 8; ++j) {
-              const uint32_t addr = rbuf + lane * 128 + (static_cast<uint32_t>(j ^ (lane & 7)) << 4);
+              const uint32_t addr = rsrc + lane * 128 + (static_cast<uint32_t>(j ^ (lane & 7)) << 4);
               asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
                            : "=r"(rq[j].x), "=r"(rq[j].y), "=r"(rq[j].z), "=r"(rq[j].w) : "r"(addr) : "memory");
             }
             __syncwarp();        // every lane has read the buffer: it may be refilled
-            if (c + c_step < c_hi) {
-              request_residual(n0 + c_step * EPI_COLS, m_base + q * 32, b);
-            } else if (have_next && s_next.kb0 == 0 && s_next.kb1 == p.k_blocks) {
-              // first chunk of the next whole tile, a main loop ahead
-              int nb2, nmt, nnt;
-              decode_tile(p, s_next.tile, nb2, nmt, nnt);
-              if (nnt * BN + c_lo * EPI_COLS < p.N)
-                request_residual(nnt * BN + c_lo * EPI_COLS, nmt * (BM * CG) + static_cast<int>(cta_rank) * BM + q * 32, nb2);
-            }
+            if (!r_shared) request_next_residual(c, c_step, c_hi, n0, m_base + q * 32, b, have_next, s_next, c_lo);
           }
           bias_s[lane] = bv0;
           bias_s[lane + 32] = bv1;
@@ -783,6 +832,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
               break;
           }
 #undef CG_EPILOGUE_CASE
+          if (ew == 0 && lane == 0 && c == c_lo) trace_event(p, TR_EPI_MATH);
           // staging buffer free again?  (the store that last used it has finished reading it) --
           // asked only now, after the arithmetic, so that the wait overlaps it
           if (lane == 0) ptx::bulk_wait_group_read<C::EPI_BUFS - 1>();
@@ -791,11 +841,14 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           stage_chunk(outw, buf_addr + lane * 128, lane);
           ptx::fence_proxy_async_smem();      // my generic-proxy writes -> visible to the TMA store
           __syncwarp();
+          if (ew == 0 && lane == 0 && c == c_lo) trace_event(p, TR_EPI_STAGED);
           if (lane == 0) {
             if (warp_rows_valid) ptx::tma_store_3d(&tmD, buf_addr, n0, m_base + q * 32, b);   // clips rows >= M, cols >= N
             ptx::bulk_commit_group();
+            if (ew == 0) trace_event(p, c == c_lo ? TR_FIRST_STORE : TR_LAST_STORE);
           }
           store_buf = (store_buf + 1 == C::EPI_BUFS) ? 0 : store_buf + 1;
+          if (r_shared) request_next_residual(c, c_step, c_hi, n0, m_base + q * 32, b, have_next, s_next, c_lo);
         }
         if (whole_tile && c_lo >= c_hi) {    // none of this warp's columns exist (ragged N): still hand the buffer back
           ptx::tc_fence_before();
@@ -817,6 +870,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         if (clock64() - t0 > (1ll << 27)) break;
     }
     if (lane == 0) ptx::bulk_wait_group<0>();   // all of this warp's stores have completed
+    if (ew == 0 && lane == 0) trace_event(p, TR_STORES_DONE);
     __syncwarp();
   }
 
@@ -830,6 +884,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   if (warp == 1) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc<CG>(tmem_base, C::TMEM_COLS);
+    if (lane == 0) trace_event(p, TR_END);
   }
 }
 

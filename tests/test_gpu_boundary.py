@@ -88,6 +88,40 @@ def test_tuning_validation_and_plan_report(cg, ctx):
     ctx.set_tuning(reset=True)
 
 
+def test_trace_records_an_ordered_timeline_and_leaves_the_result_alone(cg, ctx, oracle):
+    """cg_set_trace: per-CTA global-timer stamps of the kernel's phases, in causal order; the output is unchanged."""
+    import torch
+    p = W.make(384, 256, 512, seed=5, act=W.ACT_RELU, A=("smallint", 1.0), B=("smallint", 1.0), bias=("smallint", 1.0))
+    dev = PU.to_device(p)
+    ctx.set_tuning(reset=True)
+    ctx.set_tuning(tile_n=128, cta_group=1, num_units=6)                 # 3 x 2 whole tiles, one per CTA
+    assert cg.cg_set_trace(ctx.handle, dev["A"].data_ptr() + 4, 4) == cg.CG_ERR_INVALID_ARG   # not 8-byte aligned
+    buf = torch.zeros(8 * 32, dtype=torch.int64, device="cuda")
+    ctx.set_trace(buf, 8)
+    d = PU.run_gpu(ctx, p, dev, fill=0x7FC0)
+    ctx.set_trace(None, 0)
+    t = buf.cpu().numpy().reshape(8, 32)
+    grid = ctx.last_plan()["grid"]
+    assert grid == 6
+    START, SETUP, LD0, LDN, FULL0, MMAN, ACC, ST0, DONE, END, CLK0, CLK1 = 0, 1, 2, 3, 4, 5, 6, 9, 11, 12, 16, 17
+    for cta in range(grid):
+        r = t[cta]
+        assert r[START] > 0
+        for a, b in ((START, SETUP), (SETUP, LD0), (LD0, LDN), (LD0, FULL0), (FULL0, MMAN), (FULL0, ACC), (ACC, ST0),
+                     (ST0, DONE), (DONE, END)):
+            assert r[a] <= r[b], (cta, a, b, r[:18])
+        assert 0 < r[END] - r[START] < 1_000_000                          # well under a millisecond
+        mhz = (r[CLK1] - r[CLK0]) / (r[END] - r[START]) * 1e3
+        assert 300 < mhz < 3000, mhz
+    assert not t[grid:].any()                                             # CTAs beyond the grid wrote nothing
+    r64, r16 = PU.oracle_full(oracle, p)
+    assert PU.compare(d, r64, r16)["bit_equal"]
+    before = buf.clone()
+    PU.run_gpu(ctx, p, dev)                                               # tracing is off again
+    assert torch.equal(before, buf)
+    ctx.set_tuning(reset=True)
+
+
 def test_workspace_limit(cg):
     small = cg.Context(0, workspace_bytes=2 << 20)                       # ~1 MiB of partial-tile space
     try:
