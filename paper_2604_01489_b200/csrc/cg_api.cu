@@ -77,6 +77,7 @@ struct cg_context {
   bool log_plans = false;                // CG_LOG
   int r_shared = -1;                     // CG_R_SHARED: 0 / 1 force the residual's buffer choice (ablation), else heuristic
   int split_first = 1;                   // CG_SPLIT_FIRST=0 restores the old order (ablation)
+  int warm_up = 1;                       // CG_WARM_UP: 0 never, 1 for cluster-split plans (default), 2 always (ablation)
   unsigned long long* trace = nullptr;   // cg_set_trace
   int trace_ctas = 0;
   MapCacheEntry map_cache[MAP_CACHE_SIZE];
@@ -383,6 +384,9 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   p.stages = pl.stages;
   p.cluster_split = pl.cluster_split;
   p.r_shared = pl.r_shared;
+  // (measured: pays when the first accumulator is a long main loop away and the tail is exposed, as in
+  // the cluster split; neutral or slightly negative elsewhere)
+  p.warm_up = (h->warm_up > 1 || (h->warm_up == 1 && pl.cluster_split > 1)) ? 1 : 0;
   p.split_first = (h->split_first && pl.cluster_split <= 1 && pl.dp_units > 0 && pl.dp_units < pl.num_units) ? 1 : 0;
   p.trace = h->trace;
   p.trace_ctas = h->trace_ctas;
@@ -409,7 +413,7 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = (attr[0].val.clusterDim.x > 1 || getenv("CG_ALWAYS_CLUSTER")) ? 1 : 0;      // a plain launch when there is no cluster
   void* args[5] = {&tmA, &tmB, &tmD, &tmR, &p};
   CG_CUDA(h, cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(e.fn), args));
 
@@ -486,6 +490,7 @@ int cg_create(cg_handle_t* out, int device, size_t workspace_bytes) {
   h->log_plans = getenv("CG_LOG") != nullptr;
   if (const char* w = getenv("CG_R_SHARED")) h->r_shared = atoi(w);
   if (const char* w = getenv("CG_SPLIT_FIRST")) h->split_first = atoi(w);
+  if (const char* w = getenv("CG_WARM_UP")) h->warm_up = atoi(w);
   *out = h;
   return CG_OK;
 }

@@ -79,6 +79,7 @@ struct KernelParams {
                           // partial tiles overlaps the main loops of the whole tiles instead of ending the launch
   int stages;
   int cluster_split;      // > 1: the CTAs of a cluster of this size hold the K parts of one tile (CG == 1 only)
+  int warm_up;            // the epilogue warps first run their chunk code once without side effects (see the epilogue)
   int r_shared;           // the residual chunk lands in the output staging buffer itself (no buffers of its own)
   float alpha, beta;
   int act;
@@ -343,8 +344,32 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   const uint32_t cta_rank = (CG == 2) ? ptx::cluster_ctarank() : 0u;
   const int worker = blockIdx.x / CG;
 
+  // One k-block of A and B into ring stage `stage` (1-CTA form; the completion bytes go to `full[stage]`).
+  auto issue_loads = [&](int stage, int kb, int m0, int n0, int b, bool withhold_a) {
+    const uint32_t bar = ptx::smem_u32(&ctrl->full[stage]);
+    const uint32_t a_dst = ring_addr + stage * C::STAGE_BYTES;
+    const uint32_t b_dst = a_dst + C::A_BYTES;
+    const int k0 = kb * BK;
+    ptx::mbar_arrive_expect_tx(bar, C::STAGE_BYTES);
+    if (!withhold_a) ptx::tma_load_3d(a_dst, &tmA, bar, k0, m0, b);     // (withheld only by the starvation test hook)
+#pragma unroll
+    for (int h = 0; h < C::NSUB; ++h) {
+      const int nh = n0 + h * C::MMA_N;
+      const uint32_t dst = b_dst + h * C::SUB_B_BYTES;
+      if constexpr (B_KMAJOR) {
+        ptx::tma_load_3d(dst, &tmB, bar, k0, nh, b);
+      } else {
+#pragma unroll
+        for (int j = 0; j < C::SUB_COLS / 64; ++j)
+          ptx::tma_load_3d(dst + j * (64 * BK * 2), &tmB, bar, nh + j * 64, k0, b);
+      }
+    }
+  };
+
   // ---- set-up: barriers, tensor memory
   if (threadIdx.x == 0) {
+    ptx::prefetch_tensormap(&tmA);
+    ptx::prefetch_tensormap(&tmB);
     trace_event(p, TR_START);
     for (int s = 0; s < stages; ++s) {
       ptx::mbar_init(ptx::smem_u32(&ctrl->full[s]), 1);
@@ -356,12 +381,10 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     }
     ptx::mbar_init(ptx::smem_u32(&ctrl->drain), 1);
     for (int w = 0; w < 8; ++w) ptx::mbar_init(ptx::smem_u32(&ctrl->r_full[w]), 1);
-    ptx::prefetch_tensormap(&tmR);
     ctrl->abort = 0;
     ptx::fence_mbar_init();
-    ptx::prefetch_tensormap(&tmA);
-    ptx::prefetch_tensormap(&tmB);
     ptx::prefetch_tensormap(&tmD);
+    ptx::prefetch_tensormap(&tmR);
   }
   if (warp == 1) {
     ptx::tmem_alloc<CG>(ptx::smem_u32(&ctrl->tmem_base), C::TMEM_COLS);
@@ -400,21 +423,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           const uint32_t b_dst = a_dst + C::A_BYTES;
           const int k0 = kb * BK;
           if constexpr (CG == 1) {
-            const uint32_t bar = full0 + stage * 8;
-            ptx::mbar_arrive_expect_tx(bar, C::STAGE_BYTES);
-            if (!(p.test_starve && issued == 0)) ptx::tma_load_3d(a_dst, &tmA, bar, k0, m0, b);
-#pragma unroll
-            for (int h = 0; h < C::NSUB; ++h) {
-              const int nh = n0 + h * C::MMA_N;
-              const uint32_t dst = b_dst + h * C::SUB_B_BYTES;
-              if constexpr (B_KMAJOR) {
-                ptx::tma_load_3d(dst, &tmB, bar, k0, nh, b);
-              } else {
-#pragma unroll
-                for (int j = 0; j < C::SUB_COLS / 64; ++j)
-                  ptx::tma_load_3d(dst + j * (64 * BK * 2), &tmB, bar, nh + j * 64, k0, b);
-              }
-            }
+            issue_loads(stage, kb, m0, n0, b, p.test_starve && issued == 0);
           } else {
             // both CTAs' bytes are counted on the leader's barrier
             if (cta_rank == 0) ptx::mbar_arrive_expect_tx(full0 + stage * 8, 2 * C::STAGE_BYTES);
@@ -614,7 +623,20 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       Segment s0;
       if (peek.next(s0)) prefetch_residual(s0);
     }
-    while (ok && wi.next(s)) {
+    // Warm-up pass: until the first accumulator is ready these warps have nothing to do, and the code
+    // below has never run on this SM -- fetched on first use, from L2 or DRAM, it costs microseconds on
+    // the critical path after the last MMA of a short launch.  So the body is first run once on the
+    // worker's first segment with every wait, signal, request and store left out (it reads whatever
+    // tensor memory, shared memory and workspace hold, and writes only this warp's staging buffer).
+    int dry = p.warm_up;
+    for (;;) {
+      if (!ok) break;
+      if (dry) {
+        WorkIter peek = wi;
+        if (!peek.next(s)) break;
+      } else if (!wi.next(s)) {
+        break;
+      }
       Segment s_next;
       bool have_next = false;
       if (has_r) {               // the tile after this one: a whole main loop ahead of its use
@@ -640,7 +662,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         c_hi = (my_part + 1) * (slice_cols / EPI_COLS);
       }
       if (c_hi > n_chunks) c_hi = n_chunks;
-      if (has_r && (whole_tile || csk > 1) && !r_pending && c_lo < c_hi)
+      if (!dry && has_r && (whole_tile || csk > 1) && !r_pending && c_lo < c_hi)
         request_residual(n_base + c_lo * EPI_COLS, m_base + q * 32, b);
       // bias of this warp's columns: two values per lane and chunk, fetched before the wait for the
       // accumulator so that the loads are off the critical path
@@ -663,8 +685,8 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         bias_reg[2 * j] = b0;
         bias_reg[2 * j + 1] = b1;
       }
-      if (!wait_bar(ptx::smem_u32(&ctrl->acc_full[acc]), acc_phase, ctrl, p)) { ok = false; break; }
-      if (ew == 0 && lane == 0) trace_event(p, TR_ACC_SEEN);
+      if (!dry && !wait_bar(ptx::smem_u32(&ctrl->acc_full[acc]), acc_phase, ctrl, p)) { ok = false; break; }
+      if (!dry && ew == 0 && lane == 0) trace_event(p, TR_ACC_SEEN);
       ptx::tc_fence_after();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(acc * BN);
       const uint32_t acc_empty_bar = (CG == 2) ? ptx::mapa(ptx::smem_u32(&ctrl->acc_empty[acc]), 0)
@@ -672,7 +694,12 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 
       bool reduce = false;        // this warp must run the epilogue from workspace partials
       int first_unit = 0, last_unit = 0;
-      if (csk > 1) {
+      if (dry) {
+        if (!whole_tile && csk == 1) {       // warm the reduction of workspace partials on this unit's own slot
+          reduce = true;
+          first_unit = last_unit = s.unit;
+        }
+      } else if (csk > 1) {
         // ---- cluster split-K: exchange the partial tiles through distributed shared memory
         ptx::cluster_arrive();                 // A: every CTA of the cluster is done with its operand ring
         ptx::cluster_wait();
@@ -770,7 +797,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             ptx::tmem_ld_wait();
 #pragma unroll
             for (int j = 0; j < 32; ++j) { accv[j] = __uint_as_float(v0[j]); accv[32 + j] = __uint_as_float(v1[j]); }
-            if (c == c_hi - 1) {         // this warp's share is read: its hand-back of the buffer to the MMA warp
+            if (c == c_hi - 1 && !dry) { // this warp's share is read: its hand-back of the buffer to the MMA warp
               ptx::tc_fence_before();
               __syncwarp();
               if (lane == 0) {
@@ -792,13 +819,15 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
               }
             }
           }
-          if (ew == 0 && lane == 0 && c == c_lo) trace_event(p, TR_EPI_LOADED);
+          if (!dry && ew == 0 && lane == 0 && c == c_lo) trace_event(p, TR_EPI_LOADED);
           // residual of this chunk: this thread's row of the TMA-filled buffer (swizzled like the staging)
           uint4 rq[EPI_COLS / 8];
           if (has_r) {
-            if (!wait_bar(r_bar, r_phase, ctrl, p)) { ok = false; break; }
-            r_phase ^= 1u;
-            r_pending = false;
+            if (!dry) {
+              if (!wait_bar(r_bar, r_phase, ctrl, p)) { ok = false; break; }
+              r_phase ^= 1u;
+              r_pending = false;
+            }
             const uint32_t rsrc = r_shared ? stage_base + store_buf * EPI_BUF_BYTES : rbuf;
 #pragma unroll
             for (int j = 0; j < EPI_COLS / 8; ++j) {
@@ -807,7 +836,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                            : "=r"(rq[j].x), "=r"(rq[j].y), "=r"(rq[j].z), "=r"(rq[j].w) : "r"(addr) : "memory");
             }
             __syncwarp();        // every lane has read the buffer: it may be refilled
-            if (!r_shared) request_next_residual(c, c_step, c_hi, n0, m_base + q * 32, b, have_next, s_next, c_lo);
+            if (!r_shared && !dry) request_next_residual(c, c_step, c_hi, n0, m_base + q * 32, b, have_next, s_next, c_lo);
           }
           bias_s[lane] = bv0;
           bias_s[lane + 32] = bv1;
@@ -832,7 +861,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
               break;
           }
 #undef CG_EPILOGUE_CASE
-          if (ew == 0 && lane == 0 && c == c_lo) trace_event(p, TR_EPI_MATH);
+          if (!dry && ew == 0 && lane == 0 && c == c_lo) trace_event(p, TR_EPI_MATH);
           // staging buffer free again?  (the store that last used it has finished reading it) --
           // asked only now, after the arithmetic, so that the wait overlaps it
           if (lane == 0) ptx::bulk_wait_group_read<C::EPI_BUFS - 1>();
@@ -841,22 +870,26 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           stage_chunk(outw, buf_addr + lane * 128, lane);
           ptx::fence_proxy_async_smem();      // my generic-proxy writes -> visible to the TMA store
           __syncwarp();
-          if (ew == 0 && lane == 0 && c == c_lo) trace_event(p, TR_EPI_STAGED);
+          if (!dry && ew == 0 && lane == 0 && c == c_lo) trace_event(p, TR_EPI_STAGED);
           if (lane == 0) {
-            if (warp_rows_valid) ptx::tma_store_3d(&tmD, buf_addr, n0, m_base + q * 32, b);   // clips rows >= M, cols >= N
+            if (warp_rows_valid && !dry) ptx::tma_store_3d(&tmD, buf_addr, n0, m_base + q * 32, b);   // clips rows >= M, cols >= N
             ptx::bulk_commit_group();
-            if (ew == 0) trace_event(p, c == c_lo ? TR_FIRST_STORE : TR_LAST_STORE);
+            if (ew == 0 && !dry) trace_event(p, c == c_lo ? TR_FIRST_STORE : TR_LAST_STORE);
           }
           store_buf = (store_buf + 1 == C::EPI_BUFS) ? 0 : store_buf + 1;
-          if (r_shared) request_next_residual(c, c_step, c_hi, n0, m_base + q * 32, b, have_next, s_next, c_lo);
+          if (r_shared && !dry) request_next_residual(c, c_step, c_hi, n0, m_base + q * 32, b, have_next, s_next, c_lo);
         }
-        if (whole_tile && c_lo >= c_hi) {    // none of this warp's columns exist (ragged N): still hand the buffer back
+        if (whole_tile && c_lo >= c_hi && !dry) {    // none of this warp's columns exist (ragged N): still hand the buffer back
           ptx::tc_fence_before();
           __syncwarp();
           if (lane == 0) {
             if constexpr (CG == 2) ptx::mbar_arrive_cluster(acc_empty_bar); else ptx::mbar_arrive(acc_empty_bar);
           }
         }
+      }
+      if (dry) {
+        dry = 0;
+        continue;
       }
       if (++acc == C::ACC_BUFS) { acc = 0; acc_phase ^= 1u; }
     }
@@ -869,7 +902,9 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       while (!ptx::mbar_try_wait(r_bar, r_phase))
         if (clock64() - t0 > (1ll << 27)) break;
     }
-    if (lane == 0) ptx::bulk_wait_group<0>();   // all of this warp's stores have completed
+    // The stores have read their staging buffers: shared memory may be given up.  Their writes are
+    // complete, like every other write of the grid, when the grid is.
+    if (lane == 0) ptx::bulk_wait_group_read<0>();
     if (ew == 0 && lane == 0) trace_event(p, TR_STORES_DONE);
     __syncwarp();
   }
