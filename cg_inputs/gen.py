@@ -22,6 +22,7 @@ from __future__ import annotations
 import numpy as np
 
 TENSOR_A, TENSOR_B, TENSOR_BIAS, TENSOR_R = 1, 2, 3, 4
+TENSOR_ROW_SCALE, TENSOR_COL_SCALE = 5, 6
 
 _M64 = np.uint64(0xFFFFFFFFFFFFFFFF)
 _CHUNK = 1 << 20

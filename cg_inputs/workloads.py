@@ -4,7 +4,9 @@ ad-hoc test problems.  Pure data: no arithmetic of the method lives here.
 Activation / flag encoding of the ``act`` argument (shared by the C ABI and the oracle's C ABI):
 low byte = activation (0 none, 1 ReLU, 2 GELU-tanh, 3 SiLU, 4 GELU-erf, 5 sigmoid, 6 tanh,
 7 leaky ReLU with slope 0.01); bit 8 = B stored column-major
-([batch,N,K]); bit 9 = bias is bf16 instead of fp32.
+([batch,N,K]); bit 9 = bias is bf16 instead of fp32.  Extended entry point only: bit 10 = the bias
+is per output row (length M); bit 11 = one B shared by all batch entries; bit 12 = clamp the
+activation's result to [clamp_lo, clamp_hi].  Output dtype codes: 0 bf16, 1 fp16, 2 fp32.
 """
 from __future__ import annotations
 
@@ -20,6 +22,10 @@ ACT_NONE, ACT_RELU, ACT_GELU_TANH, ACT_SILU = 0, 1, 2, 3
 ACT_GELU_ERF, ACT_SIGMOID, ACT_TANH, ACT_LEAKY_RELU = 4, 5, 6, 7
 FLAG_B_COLMAJOR = 1 << 8
 FLAG_BIAS_BF16 = 1 << 9
+FLAG_BIAS_PER_ROW = 1 << 10
+FLAG_B_BROADCAST = 1 << 11
+FLAG_CLAMP = 1 << 12
+OUT_BF16, OUT_F16, OUT_F32 = 0, 1, 2
 
 
 @dataclass
@@ -38,6 +44,17 @@ class Problem:
     R: Optional[np.ndarray]       # uint16 bf16 bits [batch, M, N] / None
     seed: int = 0
     meta: dict = field(default_factory=dict)
+    # extended consumer family (cg_gemm_epilogue_ex); all off by default
+    row_scale: Optional[np.ndarray] = None   # float32 [M]
+    col_scale: Optional[np.ndarray] = None   # float32 [N]
+    clamp_lo: float = 0.0
+    clamp_hi: float = 0.0
+    out_dtype: int = OUT_BF16
+
+    @property
+    def extended(self) -> bool:
+        return bool(self.act & (FLAG_BIAS_PER_ROW | FLAG_B_BROADCAST | FLAG_CLAMP)) or self.row_scale is not None \
+            or self.col_scale is not None or self.out_dtype != OUT_BF16
 
     @property
     def flops(self) -> float:
@@ -46,7 +63,12 @@ class Problem:
     @property
     def algorithmic_bytes(self) -> int:
         """Each operand read once, D written once."""
-        b = 2 * self.batch * (self.M * self.K + self.K * self.N + self.M * self.N)
+        out_bytes = 4 if self.out_dtype == OUT_F32 else 2
+        b_entries = 1 if self.act & FLAG_B_BROADCAST else self.batch
+        b = 2 * self.batch * self.M * self.K + 2 * b_entries * self.K * self.N + out_bytes * self.batch * self.M * self.N
+        for v in (self.row_scale, self.col_scale):
+            if v is not None:
+                b += v.nbytes
         if self.bias is not None:
             b += self.bias.nbytes
         if self.R is not None and self.beta != 0.0:
@@ -75,23 +97,40 @@ CONFIG_ORDER = list(CONFIGS)
 
 
 def make(M, N, K, batch=1, seed=0, act=ACT_NONE, alpha=1.0, beta=0.0, A=("uniform", 1.0),
-         B=("uniform", 1.0), bias=None, R=None, name="adhoc") -> Problem:
-    """Build a problem from distribution specs (see CONFIGS for the format)."""
+         B=("uniform", 1.0), bias=None, R=None, name="adhoc", row_scale=None, col_scale=None, clamp=None,
+         out_dtype=OUT_BF16) -> Problem:
+    """Build a problem from distribution specs (see CONFIGS for the format).  ``row_scale`` /
+    ``col_scale``: distribution specs of fp32 vectors ("pow2" draws exact powers of two 2^-2..2^2);
+    ``clamp``: (lo, hi), sets FLAG_CLAMP."""
     colmajor = bool(act & FLAG_B_COLMAJOR)
     a = gen.tensor(seed, gen.TENSOR_A, (batch, M, K), A[0], A[1])
-    b = gen.tensor(seed, gen.TENSOR_B, (batch, K, N), B[0], B[1], colmajor_last2=colmajor)
+    b = gen.tensor(seed, gen.TENSOR_B, (1 if act & FLAG_B_BROADCAST else batch, K, N), B[0], B[1], colmajor_last2=colmajor)
     bias_arr = None
     if bias is not None:
         want = "bf16" if act & FLAG_BIAS_BF16 else "f32"
         dtype = bias[2] if len(bias) > 2 else want
         if dtype != want:
             raise ValueError("bias dtype does not match FLAG_BIAS_BF16")
-        bias_arr = gen.tensor(seed, gen.TENSOR_BIAS, (N,), bias[0], bias[1], dtype=dtype)
+        bias_arr = gen.tensor(seed, gen.TENSOR_BIAS, (M if act & FLAG_BIAS_PER_ROW else N,), bias[0], bias[1], dtype=dtype)
     r = None
     if R is not None:
         r = gen.tensor(seed, gen.TENSOR_R, (batch, M, N), R[0], R[1])
+
+    def scale_vec(spec, tensor_id, n):
+        if spec is None:
+            return None
+        if spec[0] == "pow2":          # exact powers of two: scaling by them commutes with every rounding
+            u = gen.tensor(seed, tensor_id, (n,), "uniform", 1.0, dtype="f32")
+            return np.exp2(np.floor((u + 1.0) * 2.5) - 2.0).astype(np.float32)
+        return gen.tensor(seed, tensor_id, (n,), spec[0], spec[1], dtype="f32")
+
+    lo, hi = clamp if clamp is not None else (0.0, 0.0)
+    if clamp is not None:
+        act |= FLAG_CLAMP
     return Problem(name=name, M=M, N=N, K=K, batch=batch, alpha=alpha, beta=beta, act=act, A=a, B=b,
-                   bias=bias_arr, R=r, seed=seed)
+                   bias=bias_arr, R=r, seed=seed, row_scale=scale_vec(row_scale, gen.TENSOR_ROW_SCALE, M),
+                   col_scale=scale_vec(col_scale, gen.TENSOR_COL_SCALE, N), clamp_lo=float(lo), clamp_hi=float(hi),
+                   out_dtype=out_dtype)
 
 
 def config(name: str) -> Problem:

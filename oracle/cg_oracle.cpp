@@ -29,6 +29,18 @@
 //   erf form (code 4); leaky ReLU has the fixed slope 0.01; the bf16 output is rounded to
 //   nearest-even directly from fp64.
 //
+// Extended consumer family (entry points *_ex; the Level-2 prompt lists "bias/add/scale",
+// "activation" and "clamp" among the consumers that follow a producer):
+//
+//     t = alpha * row_scale[m] * col_scale[n] * sum_k A[b,m,k] * B[b',k,n] + bias
+//     u = act(t);   u = min(max(u, lo), hi) when the clamp flag is set;   v = u + beta * R[b,m,n]
+//
+//   with bias = bias[n], or bias[m] under the per-row flag; b' = b, or 0 when one B is shared by all
+//   batch entries; missing scale vectors count as 1; the output is rounded once from fp64 to bf16,
+//   fp16 or fp32 (nearest-even).  With every extension off this is the formula above, bit for bit.
+//   Readings: the scales multiply the product only (like alpha), never the bias; the clamp follows the
+//   activation and precedes the residual; scale vectors and per-row bias are shared by the batch.
+//
 // Pins (tests/test_oracle_*.py): identity and all-ones operands, small-integer operands
 // against an int64 contraction, a pure-Python triple loop on tiny shapes, numpy/torch fp64
 // library routines, closed-form activation values and identities, exhaustive bf16 round
@@ -77,7 +89,34 @@ enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU_TANH = 2, ACT_SILU = 3,
        ACT_GELU_ERF = 4, ACT_SIGMOID = 5, ACT_TANH = 6, ACT_LEAKY_RELU = 7 };
 constexpr int ACT_LAST = ACT_LEAKY_RELU;
 constexpr double LEAKY_SLOPE = 0.01;
-enum { FLAG_B_COLMAJOR = 1 << 8, FLAG_BIAS_BF16 = 1 << 9 };
+enum { FLAG_B_COLMAJOR = 1 << 8, FLAG_BIAS_BF16 = 1 << 9, FLAG_BIAS_PER_ROW = 1 << 10, FLAG_B_BROADCAST = 1 << 11,
+       FLAG_CLAMP = 1 << 12 };
+enum { OUT_BF16 = 0, OUT_F16 = 1, OUT_F32 = 2 };
+
+// fp64 -> fp16 bit pattern, round to nearest, ties to even, in one rounding step.
+// fp16: 1 sign, 5 exponent (bias 15), 10 fraction bits; subnormals below 2^-14; largest finite 65504.
+inline uint16_t f64_to_f16_rne(double v) {
+  if (std::isnan(v)) return 0x7E00;
+  const uint16_t sign = std::signbit(v) ? 0x8000 : 0x0000;
+  const double a = std::fabs(v);
+  if (a == 0.0) return sign;
+  if (std::isinf(a)) return sign | 0x7C00;
+  int e;
+  std::frexp(a, &e);
+  int p = e - 1;                               // floor(log2 a)
+  if (p < -14) p = -14;
+  const double ulp = std::ldexp(1.0, p - 10);
+  const double r = std::nearbyint(a / ulp) * ulp;
+  if (r >= 65536.0) return sign | 0x7C00;       // rounded past the largest finite value
+  if (r == 0.0) return sign;
+  int er;
+  const double fr = std::frexp(r, &er);         // r = fr * 2^er, fr in [0.5, 1)
+  if (er - 1 < -14)                             // subnormal: r = frac * 2^-24
+    return sign | static_cast<uint16_t>(r / std::ldexp(1.0, -24));
+  const int biased = er - 1 + 15;
+  const uint16_t frac = static_cast<uint16_t>((fr * 2.0 - 1.0) * 1024.0);
+  return sign | static_cast<uint16_t>(biased << 10) | frac;
+}
 
 inline double activation(int act, double t) {
   switch (act) {
@@ -109,31 +148,53 @@ struct Problem {
   double alpha, beta;
   int act;
   bool b_colmajor, bias_bf16;
+  // extended family (all off in the base entry points)
+  bool bias_per_row = false, b_broadcast = false, clamp = false;
+  const float* row_scale = nullptr;   // [M] or null
+  const float* col_scale = nullptr;   // [N] or null
+  double clamp_lo = 0.0, clamp_hi = 0.0;
+  int out_dtype = OUT_BF16;
 };
 
-inline double bias_at(const Problem& p, int64_t n) {
+// bias of output (m, n): element n of the vector, or element m under the per-row flag
+inline double bias_at(const Problem& p, int64_t m, int64_t n) {
   if (!p.bias) return 0.0;
-  if (p.bias_bf16) return bf16_to_f64(static_cast<const uint16_t*>(p.bias)[n]);
-  return static_cast<double>(static_cast<const float*>(p.bias)[n]);
+  const int64_t i = p.bias_per_row ? m : n;
+  if (p.bias_bf16) return bf16_to_f64(static_cast<const uint16_t*>(p.bias)[i]);
+  return static_cast<double>(static_cast<const float*>(p.bias)[i]);
 }
 
-// B[b,k,n] through an index function: row-major [batch,K,N] or column-major [batch,N,K].
+// B[b,k,n] through an index function: row-major [batch,K,N] or column-major [batch,N,K];
+// a shared B has a single batch entry.
 inline double b_at(const Problem& p, int64_t b, int64_t k, int64_t n) {
-  const int64_t base = b * p.K * p.N;
+  const int64_t base = (p.b_broadcast ? 0 : b) * p.K * p.N;
   return bf16_to_f64(p.b_colmajor ? p.B[base + n * p.K + k] : p.B[base + k * p.N + n]);
 }
 
 inline double finish(const Problem& p, int64_t b, int64_t m, int64_t n, double s) {
-  const double t = p.alpha * s + bias_at(p, n);
-  const double u = activation(p.act, t);
+  double scale = p.alpha;
+  if (p.row_scale) scale *= static_cast<double>(p.row_scale[m]);
+  if (p.col_scale) scale *= static_cast<double>(p.col_scale[n]);
+  const double t = scale * s + bias_at(p, m, n);
+  double u = activation(p.act, t);
+  if (p.clamp) {
+    if (u < p.clamp_lo) u = p.clamp_lo;
+    if (u > p.clamp_hi) u = p.clamp_hi;
+  }
   if (p.beta != 0.0) return u + p.beta * bf16_to_f64(p.R[(b * p.M + m) * p.N + n]);
   return u;
 }
 
 // One output row (b, m): acc[n] = sum over k ascending of A[b,m,k]*B[b,k,n]; every acc[n]
 // sees the same k order as the plain m-n-k triple loop, so the two are bit-identical.
+// Stores v as element i of a typed output buffer.
+inline void put(const Problem& p, void* out, int64_t i, double v) {
+  if (p.out_dtype == OUT_F32) static_cast<float*>(out)[i] = static_cast<float>(v);       // one IEEE rounding
+  else static_cast<uint16_t*>(out)[i] = p.out_dtype == OUT_F16 ? f64_to_f16_rne(v) : f64_to_bf16_rne(v);
+}
+
 void row(const Problem& p, int64_t b, int64_t m, std::vector<double>& acc, double* out64,
-         uint16_t* out16) {
+         void* out16) {
   for (int64_t n = 0; n < p.N; ++n) acc[n] = 0.0;
   for (int64_t k = 0; k < p.K; ++k) {
     const double a = bf16_to_f64(p.A[(b * p.M + m) * p.K + k]);
@@ -142,7 +203,7 @@ void row(const Problem& p, int64_t b, int64_t m, std::vector<double>& acc, doubl
   for (int64_t n = 0; n < p.N; ++n) {
     const double v = finish(p, b, m, n, acc[n]);
     if (out64) out64[n] = v;
-    if (out16) out16[n] = f64_to_bf16_rne(v);
+    if (out16) put(p, out16, n, v);
   }
 }
 
@@ -158,6 +219,21 @@ Problem make(const void* A, const void* B, const void* bias, const void* R, int6
   p.act = act & 0xFF;
   p.b_colmajor = (act & FLAG_B_COLMAJOR) != 0;
   p.bias_bf16 = (act & FLAG_BIAS_BF16) != 0;
+  return p;
+}
+
+Problem make_ex(const void* A, const void* B, const void* bias, const void* R, int64_t M, int64_t N, int64_t K,
+                int64_t batch, double alpha, double beta, int act, const float* row_scale, const float* col_scale,
+                double clamp_lo, double clamp_hi, int out_dtype) {
+  Problem p = make(A, B, bias, R, M, N, K, batch, alpha, beta, act);
+  p.bias_per_row = (act & FLAG_BIAS_PER_ROW) != 0;
+  p.b_broadcast = (act & FLAG_B_BROADCAST) != 0;
+  p.clamp = (act & FLAG_CLAMP) != 0;
+  p.row_scale = row_scale;
+  p.col_scale = col_scale;
+  p.clamp_lo = clamp_lo;
+  p.clamp_hi = clamp_hi;
+  p.out_dtype = out_dtype;
   return p;
 }
 
@@ -220,7 +296,29 @@ int cg_ref_gemm_epilogue_points(const void* A, const void* B, const void* bias, 
   return 0;
 }
 
+// Extended family, whole problem and selected rows.  `dout` is bf16 / fp16 bit patterns (uint16) or
+// fp32 per out_dtype; row_scale / col_scale are fp32 vectors or NULL; B has one batch entry under
+// FLAG_B_BROADCAST.  rows == NULL means every row, in order.
+int cg_ref_gemm_epilogue_ex(const void* A, const void* B, const void* bias, const void* R, const int64_t* rows,
+                            int64_t nrows, double* d64, void* dout, int64_t M, int64_t N, int64_t K, int64_t batch,
+                            double alpha, double beta, int act, const float* row_scale, const float* col_scale,
+                            double clamp_lo, double clamp_hi, int out_dtype) {
+  const Problem p = make_ex(A, B, bias, R, M, N, K, batch, alpha, beta, act, row_scale, col_scale, clamp_lo, clamp_hi,
+                            out_dtype);
+  if (bad(p) || out_dtype < OUT_BF16 || out_dtype > OUT_F32 || (p.clamp && !(clamp_lo <= clamp_hi))) return 1;
+  if (!rows) nrows = batch * M;
+  const int64_t esize = out_dtype == OUT_F32 ? 4 : 2;
+  std::vector<double> acc(static_cast<size_t>(N));
+  for (int64_t i = 0; i < nrows; ++i) {
+    const int64_t r = rows ? rows[i] : i;
+    if (r < 0 || r >= batch * M) return 1;
+    row(p, r / M, r % M, acc, d64 ? d64 + i * N : nullptr, dout ? static_cast<char*>(dout) + i * N * esize : nullptr);
+  }
+  return 0;
+}
+
 // Helpers exposed so the pins can exercise them directly.
+uint16_t cg_ref_f64_to_f16(double v) { return f64_to_f16_rne(v); }
 double cg_ref_activation(int act, double t) { return activation(act & 0xFF, t); }
 uint16_t cg_ref_f64_to_bf16(double v) { return f64_to_bf16_rne(v); }
 double cg_ref_bf16_to_f64(uint16_t h) { return bf16_to_f64(h); }

@@ -19,6 +19,10 @@ ACT_NONE, ACT_RELU, ACT_GELU_TANH, ACT_SILU = 0, 1, 2, 3
 ACT_GELU_ERF, ACT_SIGMOID, ACT_TANH, ACT_LEAKY_RELU = 4, 5, 6, 7
 FLAG_B_COLMAJOR = 1 << 8
 FLAG_BIAS_BF16 = 1 << 9
+FLAG_BIAS_PER_ROW = 1 << 10
+FLAG_B_BROADCAST = 1 << 11
+FLAG_CLAMP = 1 << 12
+OUT_BF16, OUT_F16, OUT_F32 = 0, 1, 2
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "cg_oracle.cpp")
@@ -65,6 +69,11 @@ def _load():
             fn = getattr(lib, name)
             fn.argtypes = [vp, vp, vp, vp, vp, i64, vp, vp, i64, i64, i64, i64, dbl, dbl, ci]
             fn.restype = ci
+        lib.cg_ref_gemm_epilogue_ex.argtypes = [vp, vp, vp, vp, vp, i64, vp, vp, i64, i64, i64, i64, dbl, dbl, ci, vp, vp,
+                                                dbl, dbl, ci]
+        lib.cg_ref_gemm_epilogue_ex.restype = ci
+        lib.cg_ref_f64_to_f16.argtypes = [dbl]
+        lib.cg_ref_f64_to_f16.restype = ctypes.c_uint16
         lib.cg_ref_activation.argtypes = [ci, dbl]
         lib.cg_ref_activation.restype = dbl
         lib.cg_ref_f64_to_bf16.argtypes = [dbl]
@@ -131,6 +140,39 @@ def gemm_epilogue_points(A, B, bias, R, idx, M, N, K, batch, alpha, beta, act):
     if rc != 0:
         raise ValueError("oracle rejected the arguments")
     return d64, d16
+
+
+def gemm_epilogue_ex(A, B, bias, R, M, N, K, batch, alpha, beta, act, row_scale=None, col_scale=None, clamp_lo=0.0,
+                     clamp_hi=0.0, out_dtype=OUT_BF16, rows=None):
+    """Extended consumer family: scale vectors, per-row bias, clamp, shared B, bf16 / fp16 / fp32 output.
+    Returns (D64, Dout) for the whole problem ([batch,M,N]) or for ``rows`` ([len(rows),N]); Dout is
+    uint16 bit patterns (bf16, fp16) or float32."""
+    for name, x, n in (("A", A, batch * M * K), ("B", B, (1 if act & FLAG_B_BROADCAST else batch) * K * N)):
+        if x.dtype != np.uint16 or not x.flags.c_contiguous or x.size != n:
+            raise TypeError(f"{name} must be a C-contiguous uint16 (bf16 bits) array of the right size")
+    if bias is not None:
+        want = np.uint16 if act & FLAG_BIAS_BF16 else np.float32
+        if bias.dtype != want or bias.size != (M if act & FLAG_BIAS_PER_ROW else N) or not bias.flags.c_contiguous:
+            raise TypeError("bias must be a contiguous vector of the flagged dtype and length")
+    if R is not None and (R.dtype != np.uint16 or R.size != batch * M * N or not R.flags.c_contiguous):
+        raise TypeError("R must be a C-contiguous uint16 array of batch*M*N elements")
+    for name, v, n in (("row_scale", row_scale, M), ("col_scale", col_scale, N)):
+        if v is not None and (v.dtype != np.float32 or v.size != n or not v.flags.c_contiguous):
+            raise TypeError(f"{name} must be a contiguous float32 vector")
+    r = None if rows is None else np.ascontiguousarray(rows, dtype=np.int64)
+    shape = (batch, M, N) if r is None else (r.size, N)
+    d64 = np.empty(shape, dtype=np.float64)
+    dout = np.empty(shape, dtype=np.float32 if out_dtype == OUT_F32 else np.uint16)
+    rc = _load().cg_ref_gemm_epilogue_ex(_ptr(A), _ptr(B), _ptr(bias), _ptr(R), _ptr(r), 0 if r is None else r.size,
+                                         _ptr(d64), _ptr(dout), M, N, K, batch, float(alpha), float(beta), int(act),
+                                         _ptr(row_scale), _ptr(col_scale), float(clamp_lo), float(clamp_hi), int(out_dtype))
+    if rc != 0:
+        raise ValueError("oracle rejected the arguments")
+    return d64, dout
+
+
+def f64_to_f16(v):
+    return int(_load().cg_ref_f64_to_f16(float(v)))
 
 
 def activation(act, t):

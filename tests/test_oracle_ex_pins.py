@@ -1,0 +1,186 @@
+"""Pins for the oracle's extended consumer family (scale vectors, per-row bias, clamp, shared B,
+bf16 / fp16 / fp32 output).  Each check holds the oracle against something other than itself:
+exact invariants (power-of-two scaling commutes with every rounding, a clamp to one point, a
+transposed problem), closed forms, numpy's own fp64 routines and casts, and the already pinned base
+entry point where the extension must reduce to it."""
+import numpy as np
+import pytest
+
+from cg_inputs import gen, workloads as W
+
+SI = ("smallint", 1.0)
+
+
+def f64(b):
+    return gen.bf16_bits_to_f32(b).astype(np.float64)
+
+
+def run_ex(oracle, p, **kw):
+    return oracle.gemm_epilogue_ex(p.A, p.B, p.bias, p.R, p.M, p.N, p.K, p.batch, p.alpha, p.beta, p.act,
+                                   row_scale=p.row_scale, col_scale=p.col_scale, clamp_lo=p.clamp_lo, clamp_hi=p.clamp_hi,
+                                   out_dtype=p.out_dtype, **kw)
+
+
+def scaled_bits(x_bits, factor):
+    """bf16 bits times exact powers of two (broadcast), still exact in bf16 for the magnitudes used here."""
+    v = gen.bf16_bits_to_f32(x_bits) * factor.astype(np.float32)
+    b = gen.f32_to_bf16_bits(v)
+    assert np.array_equal(gen.bf16_bits_to_f32(b), v)
+    return b
+
+
+# ---------------------------------------------------------------- reduction to the base entry point
+
+@pytest.mark.parametrize("act", [W.ACT_NONE, W.ACT_SILU | W.FLAG_B_COLMAJOR, W.ACT_GELU_TANH | W.FLAG_BIAS_BF16])
+def test_extensions_off_is_the_base_entry_point(oracle, act):
+    p = W.make(37, 24, 40, batch=2, seed=3, act=act, alpha=0.75, beta=-0.5, A=("normal", 1.0), B=("normal", 0.3),
+               bias=("normal", 1.0), R=("normal", 1.0))
+    b64, b16 = oracle.gemm_epilogue(p.A, p.B, p.bias, p.R, p.M, p.N, p.K, p.batch, p.alpha, p.beta, p.act)
+    e64, e16 = run_ex(oracle, p)
+    assert np.array_equal(b64, e64) and np.array_equal(b16, e16)
+    rows = np.array([0, 5, 36, 37, 73])
+    r64, r16 = run_ex(oracle, p, rows=rows)
+    assert np.array_equal(r64, e64.reshape(-1, p.N)[rows]) and np.array_equal(r16, e16.reshape(-1, p.N)[rows])
+
+
+# ---------------------------------------------------------------- scale vectors
+
+@pytest.mark.parametrize("act", [W.ACT_NONE, W.ACT_RELU, W.ACT_LEAKY_RELU])
+@pytest.mark.parametrize("colmajor", [False, True])
+def test_power_of_two_scales_equal_prescaled_operands(oracle, act, colmajor):
+    """row_scale[m] = 2^i scales row m of A*B exactly as scaling row m of A does; col_scale[n] as
+    scaling column n of B does (a mix-up of m and n, or of rows and columns, changes the bits)."""
+    flags = W.FLAG_B_COLMAJOR if colmajor else 0
+    M, N, K, batch = 19, 24, 32, 2
+    p = W.make(M, N, K, batch, seed=9, act=act | flags, alpha=1.0, A=SI, B=SI, bias=("normal", 1.0),
+               row_scale=("pow2",), col_scale=("pow2",))
+    assert len(set(p.row_scale)) > 2 and len(set(p.col_scale)) > 2 and not np.array_equal(p.row_scale[:N][:M], p.col_scale[:M])
+    e64, e16 = run_ex(oracle, p)
+    a2 = scaled_bits(p.A, p.row_scale.reshape(1, M, 1))
+    cs = p.col_scale.reshape(1, N, 1) if colmajor else p.col_scale.reshape(1, 1, N)
+    b2 = scaled_bits(p.B, cs)
+    b64, b16 = oracle.gemm_epilogue(a2, b2, p.bias, None, M, N, K, batch, 1.0, 0.0, p.act)
+    assert np.array_equal(e64, b64) and np.array_equal(e16, b16)
+
+
+def test_scales_against_numpy_fp64(oracle):
+    M, N, K, batch = 23, 16, 48, 3
+    p = W.make(M, N, K, batch, seed=4, act=W.ACT_NONE, alpha=-1.5, beta=2.0, A=("normal", 1.0), B=("normal", 1.0),
+               bias=("normal", 1.0), R=("normal", 1.0), row_scale=("normal", 1.0), col_scale=("uniform", 2.0))
+    e64, _ = run_ex(oracle, p)
+    want = np.einsum("bmk,bkn->bmn", f64(p.A), f64(p.B)) * (p.alpha * p.row_scale.astype(np.float64)[None, :, None]
+                                                         * p.col_scale.astype(np.float64)[None, None, :])
+    want = want + p.bias.astype(np.float64)[None, None, :] + p.beta * f64(p.R)
+    assert np.allclose(e64, want, rtol=1e-12, atol=1e-12)
+
+
+def test_scales_do_not_touch_the_bias(oracle):
+    """A = 0: the product vanishes whatever the scales, so the output is act(bias) exactly."""
+    M, N, K = 9, 16, 8
+    p = W.make(M, N, K, seed=2, act=W.ACT_TANH, A=("zeros", 0.0), B=("normal", 1.0), bias=("normal", 1.0),
+               row_scale=("normal", 5.0), col_scale=("normal", 5.0))
+    e64, _ = run_ex(oracle, p)
+    assert np.allclose(e64[0], np.broadcast_to(np.tanh(p.bias.astype(np.float64)), (M, N)), rtol=1e-15, atol=0)
+
+
+# ---------------------------------------------------------------- per-row bias
+
+def test_per_row_bias_closed_form_and_transposed_problem(oracle):
+    M, N, K = 13, 24, 16
+    p = W.make(M, N, K, seed=6, act=W.ACT_SIGMOID | W.FLAG_BIAS_PER_ROW, A=("zeros", 0.0), B=("normal", 1.0), bias=("normal", 2.0))
+    assert p.bias.size == M
+    e64, _ = run_ex(oracle, p)
+    assert np.allclose(e64[0], np.broadcast_to(1.0 / (1.0 + np.exp(-p.bias.astype(np.float64)))[:, None], (M, N)), rtol=1e-15)
+    # D = A*B + bias[m]  <=>  D^T = B^T*A^T + bias[n'] : the transposed problem with an ordinary per-column bias
+    q = W.make(M, N, K, seed=7, act=W.ACT_GELU_ERF | W.FLAG_BIAS_PER_ROW, A=("normal", 1.0), B=("normal", 0.5), bias=("normal", 1.0))
+    e64, e16 = run_ex(oracle, q)
+    at = np.ascontiguousarray(np.swapaxes(q.A, 1, 2))      # [1,K,M]: A^T as the row-major right operand
+    bt = np.ascontiguousarray(np.swapaxes(q.B, 1, 2))      # [1,N,K]: B^T as the left operand
+    t64, t16 = oracle.gemm_epilogue(bt, at, q.bias, None, N, M, K, 1, 1.0, 0.0, W.ACT_GELU_ERF)
+    assert np.array_equal(np.swapaxes(t16, 1, 2), e16)
+    assert np.allclose(np.swapaxes(t64, 1, 2), e64, rtol=1e-13, atol=1e-13)    # (same products, same k order)
+
+
+# ---------------------------------------------------------------- clamp
+
+def test_clamp_invariants(oracle):
+    M, N, K = 17, 16, 24
+    base = dict(seed=8, alpha=1.0, beta=0.5, A=("normal", 1.0), B=("normal", 1.0), bias=("normal", 1.0), R=("normal", 1.0))
+    plain = W.make(M, N, K, act=W.ACT_SILU, **base)
+    p64, p16 = run_ex(oracle, plain)
+    wide = W.make(M, N, K, act=W.ACT_SILU, clamp=(-1e30, 1e30), **base)
+    w64, w16 = run_ex(oracle, wide)
+    assert np.array_equal(p64, w64) and np.array_equal(p16, w16)                  # an interval nothing leaves
+    point = W.make(M, N, K, act=W.ACT_SILU, clamp=(0.25, 0.25), **base)
+    c64, _ = run_ex(oracle, point)
+    assert np.array_equal(c64, 0.25 + 0.5 * f64(point.R))                          # one point: residual added after it
+    relu = W.make(M, N, K, act=W.ACT_RELU, **base)
+    as_clamp = W.make(M, N, K, act=W.ACT_NONE, clamp=(0.0, np.inf), **base)
+    assert np.array_equal(run_ex(oracle, relu)[0], run_ex(oracle, as_clamp)[0])    # ReLU is a clamp
+    narrow = W.make(M, N, K, act=W.ACT_NONE, clamp=(-0.5, 1.5), **base)
+    n64, _ = run_ex(oracle, narrow)
+    inner = n64 - 0.5 * f64(narrow.R)
+    assert inner.min() >= -0.5 - 1e-12 and inner.max() <= 1.5 + 1e-12 and (np.abs(inner + 0.5) < 1e-12).any() \
+        and (np.abs(inner - 1.5) < 1e-12).any()
+    with pytest.raises(ValueError):
+        run_ex(oracle, W.make(M, N, K, act=W.ACT_NONE, clamp=(1.0, -1.0), **base))
+
+
+# ---------------------------------------------------------------- shared B
+
+@pytest.mark.parametrize("colmajor", [False, True])
+def test_shared_B_equals_replicated_B(oracle, colmajor):
+    flags = W.FLAG_B_COLMAJOR if colmajor else 0
+    M, N, K, batch = 11, 16, 24, 4
+    p = W.make(M, N, K, batch, seed=5, act=W.ACT_SILU | flags | W.FLAG_B_BROADCAST, A=("normal", 1.0), B=("normal", 1.0),
+               bias=("normal", 1.0))
+    assert p.B.shape[0] == 1
+    e64, e16 = run_ex(oracle, p)
+    rep = np.ascontiguousarray(np.broadcast_to(p.B, (batch,) + p.B.shape[1:]))
+    b64, b16 = oracle.gemm_epilogue(p.A, rep, p.bias, None, M, N, K, batch, 1.0, 0.0, W.ACT_SILU | flags)
+    assert np.array_equal(e64, b64) and np.array_equal(e16, b16)
+    assert not np.array_equal(e64[0], e64[1])                                       # (the A entries do differ)
+
+
+# ---------------------------------------------------------------- output dtypes
+
+def test_fp16_rounding_exhaustive_round_trip_and_ties(oracle):
+    allbits = np.arange(65536, dtype=np.uint16)
+    vals = allbits.view(np.float16).astype(np.float64)
+    for h, v in zip(allbits.tolist(), vals.tolist()):
+        if np.isnan(v):
+            continue
+        assert oracle.f64_to_f16(v) == h, hex(h)
+    # ties go to the even neighbour; just off a tie goes to the nearer one
+    one, ulp = 1.0, 2.0 ** -10
+    assert oracle.f64_to_f16(one + ulp / 2) == 0x3C00                  # 1 + half an ulp -> 1 (even)
+    assert oracle.f64_to_f16(one + 3 * ulp / 2) == 0x3C02              # 1 + 1.5 ulp -> 1 + 2 ulp (even)
+    assert oracle.f64_to_f16(one + ulp / 2 + 1e-9) == 0x3C01
+    assert oracle.f64_to_f16(one + 3 * ulp / 2 - 1e-9) == 0x3C01
+    assert oracle.f64_to_f16(65504.0) == 0x7BFF and oracle.f64_to_f16(65519.9) == 0x7BFF
+    assert oracle.f64_to_f16(65520.0) == 0x7C00 and oracle.f64_to_f16(-1e9) == 0xFC00     # overflow to infinity
+    assert oracle.f64_to_f16(2.0 ** -25) == 0x0000 and oracle.f64_to_f16(2.0 ** -25 * 1.0001) == 0x0001
+    assert oracle.f64_to_f16(3 * 2.0 ** -25) == 0x0002                 # subnormal tie -> even
+
+
+def test_fp16_rounding_against_numpy_cast(oracle):
+    rng = np.random.default_rng(0)
+    v = np.concatenate([rng.normal(0, 1, 4000), rng.normal(0, 1e-5, 2000), rng.normal(0, 3e4, 2000),
+                        rng.uniform(-7e4, 7e4, 500)])
+    with np.errstate(over="ignore"):
+        want = v.astype(np.float16).view(np.uint16)
+    got = np.array([oracle.f64_to_f16(x) for x in v.tolist()], dtype=np.uint16)
+    assert np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("out_dtype", [W.OUT_F16, W.OUT_F32])
+def test_typed_outputs_are_one_rounding_of_the_fp64_result(oracle, out_dtype):
+    p = W.make(21, 16, 32, batch=2, seed=12, act=W.ACT_GELU_TANH, alpha=3.0, A=("normal", 1.0), B=("normal", 1.0),
+               bias=("normal", 1.0), out_dtype=out_dtype)
+    e64, eout = run_ex(oracle, p)
+    if out_dtype == W.OUT_F32:
+        assert eout.dtype == np.float32 and np.array_equal(eout, e64.astype(np.float32))
+    else:
+        assert np.array_equal(eout, e64.astype(np.float16).view(np.uint16))
+    b64, _ = oracle.gemm_epilogue(p.A, p.B, p.bias, None, p.M, p.N, p.K, p.batch, p.alpha, 0.0, p.act)
+    assert np.array_equal(b64, e64)                                                 # the dtype changes only the rounding
