@@ -327,6 +327,37 @@ def activation_sweep(ctx, p, dev, flush):
     return out
 
 
+def extended_sweep(ctx, p, dev, flush):
+    """The same problem through cg_gemm_epilogue_ex with one extension at a time: what each costs on top
+    of the base epilogue (first entry: the base entry point)."""
+    import torch
+    dvc = dev["D"].device
+    rs = torch.rand(p.M, device=dvc) + 0.5
+    cs = torch.rand(p.N, device=dvc) + 0.5
+    d16 = torch.empty((p.batch, p.M, p.N), dtype=torch.float16, device=dvc)
+    d32 = torch.empty((p.batch, p.M, p.N), dtype=torch.float32, device=dvc)
+    FLAG_CLAMP = 1 << 12
+    variants = {
+        "base": dict(),
+        "row_scale": dict(row_scale=rs),
+        "col_scale": dict(col_scale=cs),
+        "row_and_col_scale": dict(row_scale=rs, col_scale=cs),
+        "clamp": dict(act=p.act | FLAG_CLAMP, clamp_lo=-0.5, clamp_hi=2.0),
+        "out_f16": dict(D=d16, out_dtype=1),
+        "out_f32": dict(D=d32, out_dtype=2),
+    }
+    out = {}
+    for label, v in variants.items():
+        v = dict(v)
+        D = v.pop("D", dev["D"])
+        act = v.pop("act", p.act)
+        call = lambda: ctx.gemm_epilogue_ex(dev["A"], dev["B"], dev["bias"], dev["R"], D, p.M, p.N, p.K, p.batch, p.alpha, p.beta, act, **v)
+        timed(call, 2, flush)
+        out[label] = min(timed(call, 10, flush)) * 1e6
+    ctx.check()
+    return out
+
+
 def workload_table(ctx, device, peaks, names):
     """All five workloads under the heuristic plan, each launch timed alone after an L2 flush (their
     inputs may fit in L2)."""
@@ -353,6 +384,7 @@ def workload_table(ctx, device, peaks, names):
         out[name] = row
         if name == "cfg2_4096_gelu":
             out["activation_sweep_4096_us_best"] = activation_sweep(ctx, p, dev, flush)
+            out["extended_family_4096_us_best"] = extended_sweep(ctx, p, dev, flush)
         del dev
     return out
 

@@ -94,6 +94,36 @@ CG_API int cg_gemm_epilogue(cg_handle_t h, const void* A, const void* B, const v
                      int M, int N, int K, int batch, float alpha, float beta, int act, void* stream);
 
 /*
+ * The wider consumer family on the same kernel (the Level-2 optimisation prompt lists "bias/add/scale",
+ * "activation" and "clamp" among the operations to fuse into a producer's write-back):
+ *
+ *   t = alpha * row_scale[m] * col_scale[n] * sum_k A[b,m,k] * B[b',k,n] + bias
+ *   u = act(t);   u = min(max(u, clamp_lo), clamp_hi) with CG_FLAG_CLAMP;   D[b,m,n] = u + beta * R[b,m,n]
+ *
+ * Arguments as for cg_gemm_epilogue, plus, OR-ed into `act`:
+ *   CG_FLAG_BIAS_PER_ROW  bias has M entries and bias[m] is added (dtype per CG_FLAG_BIAS_BF16)
+ *   CG_FLAG_B_BROADCAST   B has a single batch entry ([K,N], or [N,K] with CG_FLAG_B_COLMAJOR) used by all (b' = 0)
+ *   CG_FLAG_CLAMP         clamp the activation's result to [ex->clamp_lo, ex->clamp_hi] (before the residual)
+ * and in *ex (NULL = all off, the call then equals cg_gemm_epilogue):
+ *   row_scale, col_scale  device, fp32 [M] / [N], or NULL (= 1); they scale the product like alpha, never the bias;
+ *                         shared by all batch entries
+ *   out_dtype             element type of D: CG_OUT_BF16, CG_OUT_F16 or CG_OUT_F32 (R stays bf16); D must be
+ *                         16-byte aligned and N % 8 == 0 as before
+ * Errors as for cg_gemm_epilogue; CG_ERR_INVALID_ARG also for clamp_lo > clamp_hi or CG_FLAG_CLAMP without ex.
+ */
+enum { CG_FLAG_BIAS_PER_ROW = 1 << 10, CG_FLAG_B_BROADCAST = 1 << 11, CG_FLAG_CLAMP = 1 << 12 };
+enum { CG_OUT_BF16 = 0, CG_OUT_F16 = 1, CG_OUT_F32 = 2 };
+typedef struct cg_epilogue_ex {
+  const float* row_scale;
+  const float* col_scale;
+  float clamp_lo, clamp_hi;
+  int out_dtype;
+} cg_epilogue_ex_t;
+CG_API int cg_gemm_epilogue_ex(cg_handle_t h, const void* A, const void* B, const void* bias, const void* R, void* D,
+                               int M, int N, int K, int batch, float alpha, float beta, int act,
+                               const cg_epilogue_ex_t* ex, void* stream);
+
+/*
  * Same operation with HOST buffers (same shapes, dtypes and layouts as above, in host memory;
  * pinned memory makes the copies asynchronous and faster).  Copies the operands to device
  * staging buffers owned by the handle (grown on demand and kept), runs the kernel, copies D

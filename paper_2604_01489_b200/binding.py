@@ -17,16 +17,25 @@ CG_ACT_NONE, CG_ACT_RELU, CG_ACT_GELU_TANH, CG_ACT_SILU = 0, 1, 2, 3
 CG_ACT_GELU_ERF, CG_ACT_SIGMOID, CG_ACT_TANH, CG_ACT_LEAKY_RELU = 4, 5, 6, 7
 CG_FLAG_B_COLMAJOR = 1 << 8
 CG_FLAG_BIAS_BF16 = 1 << 9
+CG_FLAG_BIAS_PER_ROW = 1 << 10
+CG_FLAG_B_BROADCAST = 1 << 11
+CG_FLAG_CLAMP = 1 << 12
+CG_OUT_BF16, CG_OUT_F16, CG_OUT_F32 = 0, 1, 2
 
 STATUS_NAMES = {0: "CG_OK", 1: "CG_ERR_INVALID_ARG", 2: "CG_ERR_UNSUPPORTED", 3: "CG_ERR_ARCH", 4: "CG_ERR_CUDA",
                 5: "CG_ERR_WORKSPACE", 6: "CG_ERR_TIMEOUT"}
 
-EXPORTS = ["cg_create", "cg_gemm_epilogue", "cg_gemm_epilogue_host", "cg_set_tuning", "cg_set_trace", "cg_get_last_plan",
+EXPORTS = ["cg_create", "cg_gemm_epilogue", "cg_gemm_epilogue_ex", "cg_gemm_epilogue_host", "cg_set_tuning", "cg_set_trace", "cg_get_last_plan",
            "cg_last_error", "cg_gemm_epilogue_noalloc", "cg_destroy"]
 
 
 class cg_tuning_t(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in ("tile_n", "cta_group", "num_units", "dp_units", "cluster_split", "stages", "group_m", "max_ctas")]
+
+
+class cg_epilogue_ex_t(ctypes.Structure):
+    _fields_ = [("row_scale", ctypes.c_void_p), ("col_scale", ctypes.c_void_p), ("clamp_lo", ctypes.c_float),
+                ("clamp_hi", ctypes.c_float), ("out_dtype", ctypes.c_int)]
 
 
 class cg_plan_info_t(ctypes.Structure):
@@ -65,6 +74,7 @@ def load() -> ctypes.CDLL:
     gemm_args = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, cf, cf, ci, vp]
     lib.cg_gemm_epilogue.argtypes = gemm_args
     lib.cg_gemm_epilogue_host.argtypes = gemm_args
+    lib.cg_gemm_epilogue_ex.argtypes = gemm_args[:-1] + [ctypes.POINTER(cg_epilogue_ex_t), vp]
     lib.cg_set_tuning.argtypes = [vp, ctypes.POINTER(cg_tuning_t)]
     lib.cg_set_trace.argtypes = [vp, vp, ci]
     lib.cg_get_last_plan.argtypes = [vp, ctypes.POINTER(cg_plan_info_t)]
@@ -132,6 +142,15 @@ def cg_gemm_epilogue(h, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, stre
                                    int(K), int(batch), float(alpha), float(beta), int(act), _stream_ptr(stream))
 
 
+def cg_gemm_epilogue_ex(h, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, row_scale=None, col_scale=None, clamp_lo=0.0,
+                        clamp_hi=0.0, out_dtype=CG_OUT_BF16, stream=None) -> int:
+    """The wider consumer family (scale vectors, per-row bias, clamp, shared B, bf16 / fp16 / fp32 output)."""
+    ex = cg_epilogue_ex_t(_dev_ptr(row_scale), _dev_ptr(col_scale), float(clamp_lo), float(clamp_hi), int(out_dtype))
+    return load().cg_gemm_epilogue_ex(h, _dev_ptr(A), _dev_ptr(B), _dev_ptr(bias), _dev_ptr(R), _dev_ptr(D), int(M), int(N),
+                                      int(K), int(batch), float(alpha), float(beta), int(act), ctypes.byref(ex),
+                                      _stream_ptr(stream))
+
+
 def cg_gemm_epilogue_host(h, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, stream=None) -> int:
     return load().cg_gemm_epilogue_host(h, _host_ptr(A), _host_ptr(B), _host_ptr(bias), _host_ptr(R), _host_ptr(D),
                                         int(M), int(N), int(K), int(batch), float(alpha), float(beta), int(act),
@@ -188,6 +207,11 @@ class Context:
 
     def gemm_epilogue(self, A, B, bias, R, D, M, N, K, batch=1, alpha=1.0, beta=0.0, act=CG_ACT_NONE, stream=None):
         rc = cg_gemm_epilogue(self.handle, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, stream)
+        if rc != CG_OK:
+            raise CgError(rc, cg_last_error(self.handle)[1])
+
+    def gemm_epilogue_ex(self, A, B, bias, R, D, M, N, K, batch=1, alpha=1.0, beta=0.0, act=CG_ACT_NONE, stream=None, **ex):
+        rc = cg_gemm_epilogue_ex(self.handle, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, stream=stream, **ex)
         if rc != CG_OK:
             raise CgError(rc, cg_last_error(self.handle)[1])
 

@@ -44,9 +44,10 @@ struct MapKey {
   const void* base;
   uint64_t inner, rows, batch;
   uint32_t box_inner, box_rows;
+  int dtype;
   bool operator==(const MapKey& o) const {
     return base == o.base && inner == o.inner && rows == o.rows && batch == o.batch && box_inner == o.box_inner &&
-           box_rows == o.box_rows;
+           box_rows == o.box_rows && dtype == o.dtype;
   }
 };
 struct MapCacheEntry {
@@ -152,20 +153,24 @@ int prepare_kernels(cg_context* h) {
 
 // ---- tensor maps -------------------------------------------------------------------
 
-// bf16, rank 3 (inner, rows, batch), 128-byte swizzle, zero fill outside the tensor.
+// Rank 3 (inner, rows, batch), 128-byte swizzle, zero fill outside the tensor; bf16 unless `dtype`
+// says fp16 or fp32 (output tensors of the extended entry point).
 int make_map(cg_context* h, CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows, uint64_t batch,
-             uint32_t box_inner, uint32_t box_rows) {
-  const MapKey key{base, inner, rows, batch, box_inner, box_rows};
+             uint32_t box_inner, uint32_t box_rows, int dtype = CG_OUT_BF16) {
+  const MapKey key{base, inner, rows, batch, box_inner, box_rows, dtype};
+  const uint64_t esize = dtype == CG_OUT_F32 ? 4 : 2;
+  const CUtensorMapDataType dt = dtype == CG_OUT_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                               : (dtype == CG_OUT_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
   for (int i = 0; i < MAP_CACHE_SIZE; ++i)
     if (h->map_cache[i].valid && h->map_cache[i].key == key) {
       *map = h->map_cache[i].map;
       return CG_OK;
     }
   const cuuint64_t dims[3] = {inner, rows, batch};
-  const cuuint64_t strides[2] = {inner * 2, inner * rows * 2};
+  const cuuint64_t strides[2] = {inner * esize, inner * rows * esize};
   const cuuint32_t box[3] = {box_inner, box_rows, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
-  const CUresult r = h->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box,
+  const CUresult r = h->encode(map, dt, 3, const_cast<void*>(base), dims, strides, box,
                                estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS)
@@ -185,7 +190,7 @@ size_t partial_need(long long split_units, int bn, int cgn) {
   return static_cast<size_t>(2) * split_units * cgn * BM * bn * sizeof(float);
 }
 
-int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, bool has_r, Plan* pl) {
+int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, bool has_r, Plan* pl, bool r_own_only = false) {
   const cg_tuning_t& t = h->tuning;
   const int sms = (t.max_ctas > 0 && t.max_ctas < h->num_sms) ? t.max_ctas : h->num_sms;
   const int k_blocks = ceil_div(K, BK);
@@ -310,7 +315,7 @@ int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, bool
   // The residual chunks either get buffers of their own (requested a chunk ahead of their use) or
   // land in the output staging buffers (requested after the previous store has read them): the
   // second form frees shared memory, and is taken when that buys the ring another stage.
-  pl->r_shared = (has_r && (h->r_shared >= 0 ? h->r_shared != 0 : e.stages_max > e.stages_max_r)) ? 1 : 0;
+  pl->r_shared = (has_r && !r_own_only && (h->r_shared >= 0 ? h->r_shared != 0 : e.stages_max > e.stages_max_r)) ? 1 : 0;
   const bool r_own = has_r && !pl->r_shared;
   const int smax = r_own ? e.stages_max_r : e.stages_max;       // the residual's chunk buffers cost ring depth
   int stages = t.stages > 0 ? t.stages : smax;
@@ -329,13 +334,13 @@ int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, bool
 }
 
 int validate(cg_context* h, const void* A, const void* B, const void* bias, const void* R, void* D, int M, int N,
-             int K, int batch, float beta, int act) {
+             int K, int batch, float beta, int act, int extra_flags = 0) {
   (void)bias;
   if (!h) return CG_ERR_INVALID_ARG;
   if (!A || !B || !D) return fail(h, CG_ERR_INVALID_ARG, "A, B and D must not be NULL");
   if (M < 1 || N < 1 || K < 1 || batch < 1) return fail(h, CG_ERR_INVALID_ARG, "M, N, K, batch must be >= 1");
   const int kind = act & 0xFF;
-  if (kind > CG_ACT_LEAKY_RELU || (act & ~(0xFF | CG_FLAG_B_COLMAJOR | CG_FLAG_BIAS_BF16)) != 0 || act < 0)
+  if (kind > CG_ACT_LEAKY_RELU || (act & ~(0xFF | CG_FLAG_B_COLMAJOR | CG_FLAG_BIAS_BF16 | extra_flags)) != 0 || act < 0)
     return fail(h, CG_ERR_INVALID_ARG, "unknown activation or flag bits in act=0x%x", act);
   if (beta != 0.0f && !R) return fail(h, CG_ERR_INVALID_ARG, "R must not be NULL when beta != 0");
   if (N % 8 != 0 || K % 8 != 0) return fail(h, CG_ERR_UNSUPPORTED, "N and K must be multiples of 8 (got N=%d K=%d)", N, K);
@@ -352,20 +357,24 @@ int check_alignment(cg_context* h, const void* A, const void* B, const void* bia
 }
 
 int launch(cg_context* h, const void* A, const void* B, const void* bias, const void* R, void* D, int M, int N, int K,
-           int batch, float alpha, float beta, int act, cudaStream_t stream) {
+           int batch, float alpha, float beta, int act, cudaStream_t stream, const cg_epilogue_ex_t* ex = nullptr) {
   const bool b_kmajor = (act & CG_FLAG_B_COLMAJOR) != 0;
+  const int out_dtype = ex ? ex->out_dtype : CG_OUT_BF16;
+  const bool b_broadcast = (act & CG_FLAG_B_BROADCAST) != 0;
   Plan pl;
-  int rc = make_plan(h, M, N, K, batch, b_kmajor, beta != 0.0f, &pl);
+  // (an fp32 chunk leaves through the staging buffer twice: the residual cannot land there)
+  int rc = make_plan(h, M, N, K, batch, b_kmajor, beta != 0.0f, &pl, out_dtype == CG_OUT_F32);
   if (rc != CG_OK) return rc;
   KernelEntry e;
   lookup(pl.bn, pl.cg, b_kmajor, &e);
 
   CUtensorMap tmA, tmB, tmD, tmR;
   if ((rc = make_map(h, &tmA, A, K, M, batch, BK, BM)) != CG_OK) return rc;
-  if (b_kmajor) rc = make_map(h, &tmB, B, K, N, batch, BK, e.sub_cols);
-  else rc = make_map(h, &tmB, B, N, K, batch, 64, BK);
+  const int b_entries = b_broadcast ? 1 : batch;
+  if (b_kmajor) rc = make_map(h, &tmB, B, K, N, b_entries, BK, e.sub_cols);
+  else rc = make_map(h, &tmB, B, N, K, b_entries, 64, BK);
   if (rc != CG_OK) return rc;
-  if ((rc = make_map(h, &tmD, D, N, M, batch, EPI_COLS, 32)) != CG_OK) return rc;
+  if ((rc = make_map(h, &tmD, D, N, M, batch, out_dtype == CG_OUT_F32 ? 32 : EPI_COLS, 32, out_dtype)) != CG_OK) return rc;
   if ((rc = make_map(h, &tmR, beta != 0.0f ? R : D, N, M, batch, EPI_COLS, 32)) != CG_OK) return rc;   // unused without a residual
 
   KernelParams p;
@@ -394,6 +403,17 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   p.act = act & 0xFF;
   p.bias_bf16 = (act & CG_FLAG_BIAS_BF16) ? 1 : 0;
   p.bias = bias;
+  p.bias_per_row = (act & CG_FLAG_BIAS_PER_ROW) ? 1 : 0;
+  p.b_broadcast = b_broadcast ? 1 : 0;
+  p.clamp = (act & CG_FLAG_CLAMP) ? 1 : 0;
+  p.out_dtype = out_dtype;
+  if (ex) {
+    p.clamp_lo = ex->clamp_lo;
+    p.clamp_hi = ex->clamp_hi;
+    p.row_scale = ex->row_scale;
+    p.col_scale = ex->col_scale;
+  }
+  p.ext = (p.bias_per_row || p.clamp || out_dtype != CG_OUT_BF16 || p.row_scale || p.col_scale) ? 1 : 0;
   p.R = (beta != 0.0f) ? static_cast<const __nv_bfloat16*>(R) : nullptr;
   p.partials = h->partials;
   p.tickets = h->tickets;
@@ -503,6 +523,24 @@ int cg_gemm_epilogue(cg_handle_t h, const void* A, const void* B, const void* bi
   if (rc != CG_OK) return rc;
   if ((rc = check_alignment(h, A, B, bias, R, D, beta, act)) != CG_OK) return rc;
   return launch(h, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, static_cast<cudaStream_t>(stream));
+}
+
+int cg_gemm_epilogue_ex(cg_handle_t h, const void* A, const void* B, const void* bias, const void* R, void* D, int M,
+                        int N, int K, int batch, float alpha, float beta, int act, const cg_epilogue_ex_t* ex, void* stream) {
+  if (!h) return CG_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(h->mu);
+  int rc = validate(h, A, B, bias, R, D, M, N, K, batch, beta, act, CG_FLAG_BIAS_PER_ROW | CG_FLAG_B_BROADCAST | CG_FLAG_CLAMP);
+  if (rc != CG_OK) return rc;
+  if ((rc = check_alignment(h, A, B, (act & CG_FLAG_BIAS_PER_ROW) ? nullptr : bias, R, D, beta, act)) != CG_OK) return rc;
+  if (ex) {
+    if (ex->out_dtype < CG_OUT_BF16 || ex->out_dtype > CG_OUT_F32) return fail(h, CG_ERR_INVALID_ARG, "unknown output dtype %d", ex->out_dtype);
+    if ((reinterpret_cast<uintptr_t>(ex->row_scale) | reinterpret_cast<uintptr_t>(ex->col_scale)) & 3)
+      return fail(h, CG_ERR_UNSUPPORTED, "scale vectors must be 4-byte aligned");
+    if ((act & CG_FLAG_CLAMP) && !(ex->clamp_lo <= ex->clamp_hi)) return fail(h, CG_ERR_INVALID_ARG, "clamp_lo must not exceed clamp_hi");
+  } else if (act & CG_FLAG_CLAMP) {
+    return fail(h, CG_ERR_INVALID_ARG, "CG_FLAG_CLAMP needs the bounds of a cg_epilogue_ex_t");
+  }
+  return launch(h, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, static_cast<cudaStream_t>(stream), ex);
 }
 
 int cg_gemm_epilogue_host(cg_handle_t h, const void* A, const void* B, const void* bias, const void* R, void* D, int M,

@@ -46,6 +46,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include "cg_ptx.cuh"
 
@@ -62,6 +63,7 @@ constexpr int CTRL_BYTES = 256;
 
 enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU_TANH = 2, ACT_SILU = 3,
        ACT_GELU_ERF = 4, ACT_SIGMOID = 5, ACT_TANH = 6, ACT_LEAKY_RELU = 7 };
+enum { OUT_BF16 = 0, OUT_F16 = 1, OUT_F32 = 2 };
 enum { STATUS_OK = 0, STATUS_SMEM = 4, STATUS_TIMEOUT = 6 };
 
 struct KernelParams {
@@ -85,6 +87,15 @@ struct KernelParams {
   int act;
   int bias_bf16;
   const void* bias;
+  // extended consumer family (all zero / NULL for the base entry point)
+  int ext;                // any of the following is in use
+  int bias_per_row;       // bias[m] instead of bias[n]
+  int b_broadcast;        // one B shared by all batch entries
+  int clamp;              // clamp the activation's result to [clamp_lo, clamp_hi]
+  int out_dtype;          // OUT_BF16 / OUT_F16 / OUT_F32
+  float clamp_lo, clamp_hi;
+  const float* row_scale; // fp32 [M] or NULL: multiplies alpha for row m
+  const float* col_scale; // fp32 [N] or NULL: multiplies alpha for column n
   const __nv_bfloat16* R;
   float* partials;        // [2 * (num_units - dp_units)][CG][BM * BN] fp32 partial tiles
   int* tickets;           // [num_tiles * CG * 8] (one per epilogue warp slot), zero between launches
@@ -297,6 +308,40 @@ __device__ __forceinline__ void epilogue_chunk(const float (&acc)[EPI_COLS], con
   }
 }
 
+// Extended family, one warp, one 64-column chunk, in place:
+//   t = (alpha * row_scale[m] * col_scale[n]) * acc + bias;  u = act(t);  clamp;  v = u + beta*R[m,n]
+// `row_mul` = alpha * row_scale[m]; the chunk's column scales sit two per lane (columns lane and
+// lane + 32) and are broadcast by shuffles; the bias is the chunk's column vector or this row's scalar.
+template <int ACT>
+__device__ __forceinline__ void finalize_chunk_ext(float (&acc)[EPI_COLS], const float* bias_s, float row_mul, float row_bias,
+                                                   float cs0, float cs1, const KernelParams& p, bool has_r,
+                                                   const uint4 (&rq)[EPI_COLS / 8]) {
+  const bool has_cs = p.col_scale != nullptr;
+#pragma unroll
+  for (int c = 0; c < EPI_COLS / 8; ++c) {
+    const uint32_t w[4] = {rq[c].x, rq[c].y, rq[c].z, rq[c].w};
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int col = c * 8 + j;
+      float sc = row_mul;
+      if (has_cs) sc *= __shfl_sync(0xFFFFFFFFu, col < 32 ? cs0 : cs1, col & 31);
+      const float bv = p.bias_per_row ? row_bias : bias_s[col];
+      float u = activate<ACT>(fmaf(sc, acc[col], bv));
+      if (p.clamp) u = fminf(fmaxf(u, p.clamp_lo), p.clamp_hi);
+      if (has_r) {
+        const uint32_t half = w[j >> 1];
+        u = fmaf(p.beta, __uint_as_float((j & 1) ? (half & 0xFFFF0000u) : (half << 16)), u);
+      }
+      acc[col] = u;
+    }
+  }
+}
+
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
+  __half2 h = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+
 // The packed chunk -> this thread's row of the staging buffer.  128-byte swizzle: 16-byte chunk
 // index XOR (row mod 8); staging rows are 128 B, row = lane (conflict-free, matches the D tensor map).
 __device__ __forceinline__ void stage_chunk(const uint32_t (&out)[EPI_COLS / 2], uint32_t stage_row_addr, int lane) {
@@ -345,7 +390,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   const int worker = blockIdx.x / CG;
 
   // One k-block of A and B into ring stage `stage` (1-CTA form; the completion bytes go to `full[stage]`).
-  auto issue_loads = [&](int stage, int kb, int m0, int n0, int b, bool withhold_a) {
+  auto issue_loads = [&](int stage, int kb, int m0, int n0, int b, int bb, bool withhold_a) {
     const uint32_t bar = ptx::smem_u32(&ctrl->full[stage]);
     const uint32_t a_dst = ring_addr + stage * C::STAGE_BYTES;
     const uint32_t b_dst = a_dst + C::A_BYTES;
@@ -357,11 +402,11 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       const int nh = n0 + h * C::MMA_N;
       const uint32_t dst = b_dst + h * C::SUB_B_BYTES;
       if constexpr (B_KMAJOR) {
-        ptx::tma_load_3d(dst, &tmB, bar, k0, nh, b);
+        ptx::tma_load_3d(dst, &tmB, bar, k0, nh, bb);
       } else {
 #pragma unroll
         for (int j = 0; j < C::SUB_COLS / 64; ++j)
-          ptx::tma_load_3d(dst + j * (64 * BK * 2), &tmB, bar, nh + j * 64, k0, b);
+          ptx::tma_load_3d(dst + j * (64 * BK * 2), &tmB, bar, nh + j * 64, k0, bb);
       }
     }
   };
@@ -417,13 +462,14 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         decode_tile(p, s.tile, b, mt, nt);
         const int m0 = mt * (BM * CG) + static_cast<int>(cta_rank) * BM;
         const int n0 = nt * BN + static_cast<int>(cta_rank) * C::SUB_COLS * (CG - 1);   // + h * MMA_N per sub-MMA
+        const int bb = p.b_broadcast ? 0 : b;      // batch entry of B
         for (int kb = s.kb0; kb < s.kb1; ++kb) {
           if (!wait_bar(empty0 + stage * 8, phase ^ 1u, ctrl, p)) { ok = false; break; }
           const uint32_t a_dst = ring_addr + stage * C::STAGE_BYTES;
           const uint32_t b_dst = a_dst + C::A_BYTES;
           const int k0 = kb * BK;
           if constexpr (CG == 1) {
-            issue_loads(stage, kb, m0, n0, b, p.test_starve && issued == 0);
+            issue_loads(stage, kb, m0, n0, b, bb, p.test_starve && issued == 0);
           } else {
             // both CTAs' bytes are counted on the leader's barrier
             if (cta_rank == 0) ptx::mbar_arrive_expect_tx(full0 + stage * 8, 2 * C::STAGE_BYTES);
@@ -434,11 +480,11 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
               const int nh = n0 + h * C::MMA_N;
               const uint32_t dst = b_dst + h * C::SUB_B_BYTES;
               if constexpr (B_KMAJOR) {
-                ptx::tma_load_3d_pair(dst, &tmB, bar, k0, nh, b);
+                ptx::tma_load_3d_pair(dst, &tmB, bar, k0, nh, bb);
               } else {
 #pragma unroll
                 for (int j = 0; j < C::SUB_COLS / 64; ++j)
-                  ptx::tma_load_3d_pair(dst + j * (64 * BK * 2), &tmB, bar, nh + j * 64, k0, b);
+                  ptx::tma_load_3d_pair(dst + j * (64 * BK * 2), &tmB, bar, nh + j * 64, k0, bb);
               }
             }
           }
@@ -671,7 +717,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       for (int j = 0; j < CHUNKS_PER_GROUP; ++j) {
         const int col = n_base + (c_lo + j * c_step) * EPI_COLS + lane;
         float b0 = 0.0f, b1 = 0.0f;
-        if (p.bias != nullptr) {
+        if (p.bias != nullptr && !p.bias_per_row) {
           if (p.bias_bf16) {
             const __nv_bfloat16* bp = static_cast<const __nv_bfloat16*>(p.bias);
             if (col < p.N) b0 = __bfloat162float(bp[col]);
@@ -684,6 +730,24 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         }
         bias_reg[2 * j] = b0;
         bias_reg[2 * j + 1] = b1;
+      }
+      // extended family: this row's multiplier and bias, this warp's column scales (like the bias)
+      float row_mul = p.alpha, row_bias = 0.0f;
+      float cs_reg[2 * CHUNKS_PER_GROUP];
+      if (p.ext) {
+        const int m = m_base + row_in_tile;
+        if (m < p.M) {
+          if (p.row_scale != nullptr) row_mul *= __ldg(p.row_scale + m);
+          if (p.bias_per_row && p.bias != nullptr)
+            row_bias = p.bias_bf16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(p.bias)[m])
+                                   : __ldg(static_cast<const float*>(p.bias) + m);
+        }
+#pragma unroll
+        for (int j = 0; j < CHUNKS_PER_GROUP; ++j) {
+          const int col = n_base + (c_lo + j * c_step) * EPI_COLS + lane;
+          cs_reg[2 * j] = (p.col_scale != nullptr && col < p.N) ? __ldg(p.col_scale + col) : 1.0f;
+          cs_reg[2 * j + 1] = (p.col_scale != nullptr && col + 32 < p.N) ? __ldg(p.col_scale + col + 32) : 1.0f;
+        }
       }
       if (!dry && !wait_bar(ptx::smem_u32(&ctrl->acc_full[acc]), acc_phase, ctrl, p)) { ok = false; break; }
       if (!dry && ew == 0 && lane == 0) trace_event(p, TR_ACC_SEEN);
@@ -842,6 +906,47 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           bias_s[lane + 32] = bv1;
           __syncwarp();
           uint32_t outw[EPI_COLS / 2];
+          if (p.ext) {
+#define CG_EXT_CASE(ACT) case ACT: finalize_chunk_ext<ACT>(accv, bias_s, row_mul, row_bias, cs_reg[2 * c_ord], cs_reg[2 * c_ord + 1], p, has_r, rq); break;
+            switch (p.act) {
+              CG_EXT_CASE(ACT_RELU)
+              CG_EXT_CASE(ACT_GELU_TANH)
+              CG_EXT_CASE(ACT_SILU)
+              CG_EXT_CASE(ACT_GELU_ERF)
+              CG_EXT_CASE(ACT_SIGMOID)
+              CG_EXT_CASE(ACT_TANH)
+              CG_EXT_CASE(ACT_LEAKY_RELU)
+              default: finalize_chunk_ext<ACT_NONE>(accv, bias_s, row_mul, row_bias, cs_reg[2 * c_ord], cs_reg[2 * c_ord + 1], p, has_r, rq); break;
+            }
+#undef CG_EXT_CASE
+            if (p.out_dtype == OUT_F32) {
+              // fp32 rows are 256 bytes: the chunk leaves as two 32-column boxes through the same buffer
+#pragma unroll
+              for (int hh = 0; hh < 2; ++hh) {
+                if (lane == 0) ptx::bulk_wait_group_read<C::EPI_BUFS - 1>();
+                __syncwarp();
+                const uint32_t buf_addr = stage_base + store_buf * EPI_BUF_BYTES;
+#pragma unroll
+                for (int cc = 0; cc < 8; ++cc) {
+                  const uint32_t addr = buf_addr + lane * 128 + (static_cast<uint32_t>(cc ^ (lane & 7)) << 4);
+                  const float* v = accv + hh * 32 + cc * 4;
+                  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(__float_as_uint(v[0])),
+                               "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])) : "memory");
+                }
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                  if (warp_rows_valid && !dry && n0 + hh * 32 < p.N) ptx::tma_store_3d(&tmD, buf_addr, n0 + hh * 32, m_base + q * 32, b);
+                  ptx::bulk_commit_group();
+                }
+                store_buf = (store_buf + 1 == C::EPI_BUFS) ? 0 : store_buf + 1;
+              }
+              continue;
+            }
+#pragma unroll
+            for (int i = 0; i < EPI_COLS / 2; ++i)
+              outw[i] = p.out_dtype == OUT_F16 ? pack_f16x2(accv[2 * i], accv[2 * i + 1]) : pack_bf16x2(accv[2 * i], accv[2 * i + 1]);
+          } else {
 #define CG_EPILOGUE_CASE(ACT)                                                              \
   case ACT:                                                                                \
     if (has_r) epilogue_chunk<ACT, true>(accv, bias_s, p.alpha, p.beta, rq, outw);         \
@@ -861,6 +966,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
               break;
           }
 #undef CG_EPILOGUE_CASE
+          }
           if (!dry && ew == 0 && lane == 0 && c == c_lo) trace_event(p, TR_EPI_MATH);
           // staging buffer free again?  (the store that last used it has finished reading it) --
           // asked only now, after the arithmetic, so that the wait overlaps it

@@ -58,3 +58,68 @@ def oracle_full(oracle, p):
 
 def oracle_rows(oracle, p, rows):
     return oracle.gemm_epilogue_rows(p.A, p.B, p.bias, p.R, rows, p.M, p.N, p.K, p.batch, p.alpha, p.beta, p.act)
+
+
+# ------------------------------------------------------------------ extended consumer family
+
+def to_device_ex(p, device="cuda:0"):
+    """Like to_device, with the scale vectors and an output buffer of the problem's dtype."""
+    import torch
+    dev = to_device(p, device)
+    dev["row_scale"] = None if p.row_scale is None else torch.from_numpy(p.row_scale).to(device)
+    dev["col_scale"] = None if p.col_scale is None else torch.from_numpy(p.col_scale).to(device)
+    dt = {W.OUT_BF16: torch.bfloat16, W.OUT_F16: torch.float16, W.OUT_F32: torch.float32}[p.out_dtype]
+    dev["D"] = torch.empty((p.batch, p.M, p.N), dtype=dt, device=device)
+    return dev
+
+
+def run_gpu_ex(ctx, p, dev=None, fill_nan=True):
+    """One cg_gemm_epilogue_ex call; returns D as raw bits (uint16) or float32 values [batch, M, N]."""
+    import torch
+    if dev is None:
+        dev = to_device_ex(p)
+    if fill_nan:
+        dev["D"].fill_(float("nan"))
+    ctx.gemm_epilogue_ex(dev["A"], dev["B"], dev["bias"], dev["R"], dev["D"], p.M, p.N, p.K, p.batch, p.alpha, p.beta, p.act,
+                         row_scale=dev["row_scale"], col_scale=dev["col_scale"], clamp_lo=p.clamp_lo, clamp_hi=p.clamp_hi,
+                         out_dtype=p.out_dtype)
+    ctx.check()
+    if p.out_dtype == W.OUT_F32:
+        return dev["D"].cpu().numpy()
+    return dev["D"].view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def oracle_ex(oracle, p, rows=None):
+    return oracle.gemm_epilogue_ex(p.A, p.B, p.bias, p.R, p.M, p.N, p.K, p.batch, p.alpha, p.beta, p.act,
+                                   row_scale=p.row_scale, col_scale=p.col_scale, clamp_lo=p.clamp_lo, clamp_hi=p.clamp_hi,
+                                   out_dtype=p.out_dtype, rows=rows)
+
+
+def typed_to_f64(d, out_dtype):
+    if out_dtype == W.OUT_F32:
+        return d.astype(np.float64)
+    if out_dtype == W.OUT_F16:
+        return d.view(np.float16).astype(np.float64)
+    return gen.bf16_bits_to_f32(d).astype(np.float64)
+
+
+# fp32 output keeps the fp32 accumulator's accuracy: a tolerance fifty times tighter than for 16-bit outputs
+ELEM_TOL_F32 = 2e-4
+FRO_TOL_F32 = 1e-4
+
+
+def compare_ex(d, ref64, refout, out_dtype):
+    """Error figures of a typed GPU result against the oracle's fp64 result; bit equality against its typed one."""
+    got = typed_to_f64(d, out_dtype).reshape(ref64.shape)
+    etol, ftol = (ELEM_TOL_F32, FRO_TOL_F32) if out_dtype == W.OUT_F32 else (ELEM_TOL, FRO_TOL)
+    err = np.abs(got - ref64)
+    bound = etol * (np.abs(ref64) + 1.0)
+    nref = float(np.linalg.norm(ref64))
+    fro = float(np.linalg.norm(got - ref64) / nref) if nref > 0 else float(np.max(np.abs(got)))
+    out = dict(worst_ratio=float(np.max(err / bound)) if err.size else 0.0, rel_fro=fro, n_bad=int(np.sum(~(err <= bound))),
+               finite=bool(np.all(np.isfinite(got))))
+    same = d.reshape(refout.shape) == refout
+    out["bit_equal"] = bool(np.all(same))
+    out["n_bits_differ"] = int(np.sum(~same))
+    out["ok"] = out["finite"] and out["n_bad"] == 0 and fro <= ftol
+    return out

@@ -1,0 +1,158 @@
+"""GPU parity of the extended consumer family (cg_gemm_epilogue_ex) against the CPU oracle on the same
+seeded inputs.  Integer-valued operands, power-of-two scales and a linear / ReLU / clamp epilogue make
+every fp32 intermediate exact, so the typed output must match the oracle's bit for bit; everything else
+must satisfy |D_gpu - D_ref| <= tol * (|D_ref| + 1) elementwise and a relative Frobenius bound against
+the oracle's fp64 result (tol 1e-2 / 5e-3 for 16-bit outputs, 2e-4 / 1e-4 for fp32 output)."""
+import numpy as np
+import pytest
+
+from cg_inputs import workloads as W
+
+import parity_util as PU
+
+pytestmark = pytest.mark.gpu
+
+SI = ("smallint", 1.0)
+P2 = ("pow2",)
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device")
+    import paper_2604_01489_b200 as cg
+    c = cg.Context(0)
+    yield c
+    c.close()
+
+
+def check(ctx, oracle, p, exact=False, **tuning):
+    ctx.set_tuning(reset=True)
+    if tuning:
+        ctx.set_tuning(**tuning)
+    d = PU.run_gpu_ex(ctx, p)                     # D pre-filled with NaNs: every element must be written
+    r64, rout = PU.oracle_ex(oracle, p)
+    c = PU.compare_ex(d, r64, rout, p.out_dtype)
+    assert c["finite"], "an output element was not written or is not finite"
+    assert c["ok"], c
+    if exact:
+        assert c["bit_equal"], c
+    return ctx.last_plan()
+
+
+PLANS = [dict(tile_n=64, cta_group=1), dict(tile_n=128, cta_group=1), dict(tile_n=256, cta_group=1),
+         dict(tile_n=128, cta_group=2), dict(tile_n=256, cta_group=2), dict(tile_n=512, cta_group=2), dict()]
+SHAPES = [(129, 136, 200, 1), (200, 264, 72, 3), (384, 512, 256, 1), (77, 1000, 136, 2)]
+
+
+@pytest.mark.parametrize("out_dtype", [W.OUT_BF16, W.OUT_F16, W.OUT_F32], ids=["bf16", "f16", "f32"])
+@pytest.mark.parametrize("plan", PLANS, ids=lambda d: "auto" if not d else f"bn{d['tile_n']}cg{d['cta_group']}")
+@pytest.mark.parametrize("shape", SHAPES, ids=lambda s: "x".join(map(str, s)))
+def test_everything_on_integer_operands_bit_exact(ctx, oracle, shape, plan, out_dtype):
+    """Scale vectors, per-row bias, clamp, shared column-major B and a residual at once."""
+    M, N, K, batch = shape
+    act = W.ACT_RELU | W.FLAG_B_COLMAJOR | W.FLAG_BIAS_PER_ROW | W.FLAG_B_BROADCAST
+    p = W.make(M, N, K, batch, seed=M + N, act=act, alpha=2.0, beta=-1.0, A=SI, B=SI, bias=SI, R=SI, row_scale=P2,
+               col_scale=P2, clamp=(0.0, 96.0), out_dtype=out_dtype)
+    check(ctx, oracle, p, exact=True, **plan)
+
+
+@pytest.mark.parametrize("feature", ["row_scale", "col_scale", "bias_row", "bias_row_bf16", "clamp", "shared_b", "none"])
+@pytest.mark.parametrize("out_dtype", [W.OUT_BF16, W.OUT_F32], ids=["bf16", "f32"])
+def test_each_feature_alone_bit_exact(ctx, oracle, feature, out_dtype):
+    kw = dict(act=W.ACT_NONE, alpha=1.0, beta=0.0, A=SI, B=SI, bias=SI, R=None, out_dtype=out_dtype)
+    if feature == "row_scale":
+        kw["row_scale"] = P2
+    elif feature == "col_scale":
+        kw["col_scale"] = P2
+    elif feature == "bias_row":
+        kw["act"] |= W.FLAG_BIAS_PER_ROW
+    elif feature == "bias_row_bf16":
+        kw["act"] |= W.FLAG_BIAS_PER_ROW | W.FLAG_BIAS_BF16
+    elif feature == "clamp":
+        kw["clamp"] = (-20.0, 33.0)
+    elif feature == "shared_b":
+        kw["act"] |= W.FLAG_B_BROADCAST
+    elif out_dtype == W.OUT_BF16:
+        pytest.skip("nothing extended: covered by the base entry point's tests")
+    p = W.make(300, 328, 512, batch=2, seed=21, **kw)
+    assert p.extended
+    check(ctx, oracle, p, exact=True)
+    check(ctx, oracle, p, exact=True, tile_n=128, cta_group=1, num_units=29)        # stream-K, reduced from the workspace
+    check(ctx, oracle, p, exact=True, tile_n=128, cta_group=1, cluster_split=2)     # split across a cluster
+
+
+@pytest.mark.parametrize("act", [W.ACT_NONE, W.ACT_RELU, W.ACT_GELU_TANH, W.ACT_SILU, W.ACT_GELU_ERF, W.ACT_SIGMOID, W.ACT_TANH,
+                                 W.ACT_LEAKY_RELU])
+@pytest.mark.parametrize("out_dtype", [W.OUT_BF16, W.OUT_F16, W.OUT_F32], ids=["bf16", "f16", "f32"])
+def test_random_inputs_every_activation(ctx, oracle, act, out_dtype):
+    p = W.make(333, 520, 456, batch=2, seed=act * 3 + out_dtype, act=act | W.FLAG_BIAS_BF16, alpha=0.7, beta=0.5,
+               A=("normal", 1.0), B=("normal", 0.08), bias=("normal", 1.0), R=("normal", 1.0), row_scale=("uniform", 2.0),
+               col_scale=("normal", 1.0), clamp=(-0.75, 1.25), out_dtype=out_dtype)
+    check(ctx, oracle, p)
+    check(ctx, oracle, p, tile_n=256, cta_group=2)
+
+
+def test_ragged_edges_and_tiny_shapes(ctx, oracle):
+    for (M, N, K, batch) in [(1, 8, 8, 1), (127, 72, 8, 2), (33, 40, 1032, 1)]:
+        for out_dtype in (W.OUT_F16, W.OUT_F32):
+            p = W.make(M, N, K, batch, seed=M, act=W.ACT_RELU | W.FLAG_BIAS_PER_ROW, A=SI, B=SI, bias=SI, R=SI, beta=1.0,
+                       row_scale=P2, col_scale=P2, out_dtype=out_dtype)
+            check(ctx, oracle, p, exact=True)
+
+
+def test_null_descriptor_is_the_base_entry_point(ctx, oracle):
+    import torch
+    import paper_2604_01489_b200 as cg
+    p = W.make(200, 264, 136, batch=2, seed=5, act=W.ACT_SILU, alpha=0.5, beta=1.0, A=("normal", 1.0), B=("normal", 0.1),
+               bias=("normal", 1.0), R=("normal", 1.0))
+    dev = PU.to_device(p)
+    ctx.set_tuning(reset=True)
+    base = PU.run_gpu(ctx, p, dev, fill=0x7FC0).copy()
+    dev["D"].view(torch.int16).fill_(0x7FC0)
+    lib = cg.load()
+    rc = lib.cg_gemm_epilogue_ex(ctx.handle, dev["A"].data_ptr(), dev["B"].data_ptr(), dev["bias"].data_ptr(), dev["R"].data_ptr(),
+                                 dev["D"].data_ptr(), p.M, p.N, p.K, p.batch, p.alpha, p.beta, p.act, None,
+                                 torch.cuda.current_stream().cuda_stream)
+    assert rc == cg.CG_OK
+    ctx.check()
+    assert np.array_equal(dev["D"].view(torch.int16).cpu().numpy().view(np.uint16), base)
+
+
+def test_error_codes(ctx):
+    import torch
+    import paper_2604_01489_b200 as cg
+    p = W.make(64, 64, 64, seed=1)
+    dev = PU.to_device(p)
+    dev["D"].view(torch.int16).fill_(0x1234)
+    h = ctx.handle
+    call = lambda act=0, **ex: cg.cg_gemm_epilogue_ex(h, dev["A"], dev["B"], None, None, dev["D"], 64, 64, 64, 1, 1.0, 0.0, act, **ex)
+    assert call(act=cg.CG_FLAG_CLAMP, clamp_lo=1.0, clamp_hi=-1.0) == cg.CG_ERR_INVALID_ARG
+    assert call(out_dtype=3) == cg.CG_ERR_INVALID_ARG and call(out_dtype=-1) == cg.CG_ERR_INVALID_ARG
+    assert call(act=1 << 13) == cg.CG_ERR_INVALID_ARG
+    assert call(row_scale=dev["A"].data_ptr() + 2) == cg.CG_ERR_UNSUPPORTED
+    # the base entry point does not know the extended flags
+    assert cg.cg_gemm_epilogue(h, dev["A"], dev["B"], None, None, dev["D"], 64, 64, 64, 1, 1.0, 0.0, cg.CG_FLAG_CLAMP) == cg.CG_ERR_INVALID_ARG
+    lib = cg.load()
+    rc = lib.cg_gemm_epilogue_ex(h, dev["A"].data_ptr(), dev["B"].data_ptr(), None, None, dev["D"].data_ptr(), 64, 64, 64, 1, 1.0, 0.0,
+                                 cg.CG_FLAG_CLAMP, None, torch.cuda.current_stream().cuda_stream)
+    assert rc == cg.CG_ERR_INVALID_ARG                                   # a clamp without its bounds
+    torch.cuda.synchronize()
+    assert bool((dev["D"].view(torch.int16) == 0x1234).all()), "D was written by a rejected call"
+    assert call(act=cg.CG_FLAG_CLAMP, clamp_lo=-1.0, clamp_hi=1.0) == cg.CG_OK
+    ctx.check()
+
+
+def test_full_size_shared_weight_sampled(ctx, oracle):
+    """A batched projection with one shared weight at a bench-like size, checked on sampled rows."""
+    p = W.make(1024, 1024, 1024, batch=8, seed=31, act=W.ACT_GELU_ERF | W.FLAG_B_BROADCAST, alpha=1.0, beta=1.0,
+               A=("normal", 1.0), B=("normal", 1.0 / 32.0), bias=("normal", 0.1), R=("normal", 1.0), col_scale=("uniform", 1.0),
+               clamp=(-1.0, 3.0), out_dtype=W.OUT_F16)
+    ctx.set_tuning(reset=True)
+    d = PU.run_gpu_ex(ctx, p)
+    rows = W.sample_rows(p, 48)
+    r64, rout = PU.oracle_ex(oracle, p, rows=rows)
+    c = PU.compare_ex(d.reshape(-1, p.N)[rows], r64, rout, p.out_dtype)
+    assert c["ok"], c
+    assert np.isfinite(PU.typed_to_f64(d, p.out_dtype)).all()
