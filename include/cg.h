@@ -179,6 +179,8 @@ typedef struct cg_plan_info {
   int smem_bytes;  /* dynamic shared memory per CTA          */
   int launches;    /* kernels launched by the call (always 1)*/
   int cluster_split; /* K parts per tile held by one cluster (1 = off) */
+  int latency_kernel; /* 1: the short single-tile-per-CTA kernel for small problems ran (every tile on its own SM,
+                         K <= 512, at most 2^19 outputs, base epilogue, no plan override) */
 } cg_plan_info_t;
 CG_API int cg_get_last_plan(cg_handle_t h, cg_plan_info_t* out);
 

@@ -40,7 +40,8 @@ class cg_epilogue_ex_t(ctypes.Structure):
 
 class cg_plan_info_t(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in ("tile_m", "tile_n", "cta_group", "stages", "group_m", "grid", "num_tiles",
-                                            "num_units", "dp_units", "k_blocks", "smem_bytes", "launches", "cluster_split")]
+                                            "num_units", "dp_units", "k_blocks", "smem_bytes", "launches", "cluster_split",
+                                            "latency_kernel")]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}

@@ -14,6 +14,7 @@
 #include <mutex>
 
 #include "cg_kernel.cuh"
+#include "cg_small.cuh"
 
 namespace {
 
@@ -78,6 +79,7 @@ struct cg_context {
   bool log_plans = false;                // CG_LOG
   int r_shared = -1;                     // CG_R_SHARED: 0 / 1 force the residual's buffer choice (ablation), else heuristic
   int split_first = 1;                   // CG_SPLIT_FIRST=0 restores the old order (ablation)
+  int small_kernel = 1;                  // CG_SMALL=0: never take the latency kernel (ablation)
   int warm_up = 1;                       // CG_WARM_UP: 0 never, 1 for cluster-split plans (default), 2 always (ablation)
   unsigned long long* trace = nullptr;   // cg_set_trace
   int trace_ctas = 0;
@@ -138,6 +140,20 @@ bool lookup(int bn, int cgn, bool km, KernelEntry* out) {
   return false;
 }
 
+typedef void (*SmallKernelFn)(const CUtensorMap, const CUtensorMap, const SmallParams);
+SmallKernelFn small_kernel_for(int act) {
+  switch (act) {
+    case CG_ACT_RELU: return small_gemm_kernel<ACT_RELU>;
+    case CG_ACT_GELU_TANH: return small_gemm_kernel<ACT_GELU_TANH>;
+    case CG_ACT_SILU: return small_gemm_kernel<ACT_SILU>;
+    case CG_ACT_GELU_ERF: return small_gemm_kernel<ACT_GELU_ERF>;
+    case CG_ACT_SIGMOID: return small_gemm_kernel<ACT_SIGMOID>;
+    case CG_ACT_TANH: return small_gemm_kernel<ACT_TANH>;
+    case CG_ACT_LEAKY_RELU: return small_gemm_kernel<ACT_LEAKY_RELU>;
+    default: return small_gemm_kernel<ACT_NONE>;
+  }
+}
+
 int prepare_kernels(cg_context* h) {
   const int bns[4] = {64, 128, 256, 512};
   for (int cgn = 1; cgn <= 2; ++cgn)
@@ -148,6 +164,9 @@ int prepare_kernels(cg_context* h) {
         CG_CUDA(h, cudaFuncSetAttribute(reinterpret_cast<const void*>(e.fn), cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         SMEM_LIMIT));
       }
+  for (int act = 0; act <= CG_ACT_LEAKY_RELU; ++act)
+    CG_CUDA(h, cudaFuncSetAttribute(reinterpret_cast<const void*>(small_kernel_for(act)), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    SMALL_MAX_KB * SMALL_STAGE_BYTES + 1024));
   return CG_OK;
 }
 
@@ -356,9 +375,63 @@ int check_alignment(cg_context* h, const void* A, const void* B, const void* bia
   return CG_OK;
 }
 
+// Small problems (every tile on its own SM, K of at most 512, base epilogue, no plan override) go to
+// the latency kernel.  Returns CG_OK after launching, or -1 when the problem is not one of those.
+int launch_small(cg_context* h, const void* A, const void* B, const void* bias, const void* R, void* D, int M, int N, int K,
+                 int batch, float alpha, float beta, int act, cudaStream_t stream) {
+  const cg_tuning_t& t = h->tuning;
+  if (!h->small_kernel || t.tile_n || t.cta_group || t.num_units || t.dp_units || t.cluster_split || t.stages || t.group_m ||
+      t.max_ctas)
+    return -1;
+  const int k_blocks = ceil_div(K, BK);
+  const long long tiles = static_cast<long long>(batch) * ceil_div(M, BM) * ceil_div(N, SMALL_BN);
+  if (k_blocks > SMALL_MAX_KB || tiles > h->num_sms || static_cast<long long>(batch) * M * N > (1ll << 19)) return -1;
+  const bool b_kmajor = (act & CG_FLAG_B_COLMAJOR) != 0;
+  CUtensorMap tmA, tmB;
+  int rc;
+  if ((rc = make_map(h, &tmA, A, K, M, batch, BK, BM)) != CG_OK) return rc;
+  if (b_kmajor) rc = make_map(h, &tmB, B, K, N, batch, BK, SMALL_BN);
+  else rc = make_map(h, &tmB, B, N, K, batch, SMALL_BN, BK);
+  if (rc != CG_OK) return rc;
+  SmallParams p;
+  memset(&p, 0, sizeof p);
+  p.M = M; p.N = N; p.K = K; p.batch = batch;
+  p.tiles_m = ceil_div(M, BM); p.tiles_n = ceil_div(N, SMALL_BN); p.k_blocks = k_blocks;
+  p.alpha = alpha; p.beta = beta;
+  p.act = act & 0xFF;
+  p.bias_bf16 = (act & CG_FLAG_BIAS_BF16) ? 1 : 0;
+  p.b_kmajor = b_kmajor ? 1 : 0;
+  p.bias = bias;
+  p.R = (beta != 0.0f) ? static_cast<const __nv_bfloat16*>(R) : nullptr;
+  p.D = static_cast<__nv_bfloat16*>(D);
+  p.status = h->status;
+  p.wait_limit = h->wait_limit;
+  p.test_starve = h->test_starve;
+  p.trace = h->trace;
+  p.trace_ctas = h->trace_ctas;
+  const int smem = k_blocks * SMALL_STAGE_BYTES + 1024;
+  small_kernel_for(p.act)<<<static_cast<unsigned>(tiles), 128, smem, stream>>>(tmA, tmB, p);
+  CG_CUDA(h, cudaGetLastError());
+  cg_plan_info_t& lp = h->last_plan;
+  memset(&lp, 0, sizeof lp);
+  lp.tile_m = BM; lp.tile_n = SMALL_BN; lp.cta_group = 1; lp.stages = k_blocks; lp.group_m = 1;
+  lp.grid = static_cast<int>(tiles); lp.num_tiles = lp.grid; lp.num_units = lp.grid; lp.dp_units = lp.grid;
+  lp.k_blocks = k_blocks; lp.smem_bytes = smem; lp.launches = 1; lp.cluster_split = 1; lp.latency_kernel = 1;
+  h->last_status = CG_OK;
+  h->last_msg[0] = 0;
+  if (h->log_plans) fprintf(stderr, "[cg] M=%d N=%d K=%d batch=%d latency kernel, grid=%d smem=%d\n", M, N, K, batch, lp.grid, smem);
+  return CG_OK;
+}
+
 int launch(cg_context* h, const void* A, const void* B, const void* bias, const void* R, void* D, int M, int N, int K,
            int batch, float alpha, float beta, int act, cudaStream_t stream, const cg_epilogue_ex_t* ex = nullptr) {
   const bool b_kmajor = (act & CG_FLAG_B_COLMAJOR) != 0;
+  const bool ext_in_use = (act & (CG_FLAG_BIAS_PER_ROW | CG_FLAG_B_BROADCAST | CG_FLAG_CLAMP)) != 0 ||
+                          (ex && (ex->row_scale || ex->col_scale || ex->out_dtype != CG_OUT_BF16));
+  if (!ext_in_use) {
+    const int rs = launch_small(h, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, stream);
+    if (rs >= 0) return rs;
+  }
   const int out_dtype = ex ? ex->out_dtype : CG_OUT_BF16;
   const bool b_broadcast = (act & CG_FLAG_B_BROADCAST) != 0;
   Plan pl;
@@ -441,7 +514,7 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   lp.tile_m = BM * pl.cg; lp.tile_n = pl.bn; lp.cta_group = pl.cg; lp.stages = pl.stages; lp.group_m = pl.group_m;
   lp.grid = pl.grid; lp.num_tiles = pl.num_tiles; lp.num_units = pl.num_units; lp.dp_units = pl.dp_units;
   lp.k_blocks = pl.k_blocks;
-  lp.smem_bytes = pl.smem; lp.launches = 1; lp.cluster_split = pl.cluster_split;
+  lp.smem_bytes = pl.smem; lp.launches = 1; lp.cluster_split = pl.cluster_split; lp.latency_kernel = 0;
   h->last_status = CG_OK;
   h->last_msg[0] = 0;
   if (h->log_plans)
@@ -511,6 +584,7 @@ int cg_create(cg_handle_t* out, int device, size_t workspace_bytes) {
   if (const char* w = getenv("CG_R_SHARED")) h->r_shared = atoi(w);
   if (const char* w = getenv("CG_SPLIT_FIRST")) h->split_first = atoi(w);
   if (const char* w = getenv("CG_WARM_UP")) h->warm_up = atoi(w);
+  if (const char* w = getenv("CG_SMALL")) h->small_kernel = atoi(w);
   *out = h;
   return CG_OK;
 }

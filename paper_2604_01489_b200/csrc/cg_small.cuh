@@ -1,0 +1,230 @@
+// Latency kernel for small problems: one CTA per 128 x 64 output tile, every k-block of the tile
+// resident in shared memory (K <= 512), no persistent loop, no split, and code kept short on
+// purpose -- on a cold launch the instructions themselves come from DRAM, and for a problem of a
+// few microseconds the length of the executed path is what the launch costs.
+//
+//   D[b,m,n] = act( alpha * sum_k A[b,m,k] * B[b,k,n] + bias[n] ) + beta * R[b,m,n]
+//
+// 128 threads.  Thread 0 initialises the barriers, issues all TMA loads at once (one `full`
+// barrier per k-block) and then issues the tcgen05.mma sequence as the k-blocks land; warp 1
+// allocates tensor memory.  All four warps run the epilogue: warp w owns accumulator rows
+// 32w..32w+31 (its TMEM lane quarter), sixteen columns at a time: TMEM -> registers, bias (two
+// columns per lane, broadcast by shuffles), activation (a template parameter), residual
+// and output straight from / to global memory (32 bytes per thread and step).  Waits are bounded as
+// in the main kernel.
+#pragma once
+
+#include "cg_kernel.cuh"
+
+namespace cg {
+
+constexpr int SMALL_BN = 64;
+constexpr int SMALL_MAX_KB = 8;
+constexpr int SMALL_A_BYTES = BM * BK * 2;
+constexpr int SMALL_B_BYTES = SMALL_BN * BK * 2;
+constexpr int SMALL_STAGE_BYTES = SMALL_A_BYTES + SMALL_B_BYTES;
+constexpr int SMALL_TMEM_COLS = 64;
+
+struct SmallParams {
+  int M, N, K, batch;
+  int tiles_m, tiles_n, k_blocks;
+  float alpha, beta;
+  int act, bias_bf16, b_kmajor;
+  const void* bias;
+  const __nv_bfloat16* R;
+  __nv_bfloat16* D;
+  int* status;
+  long long wait_limit;
+  int test_starve;
+  unsigned long long* trace;   // debug timeline (see cg_set_trace), or NULL
+  int trace_ctas;
+};
+
+struct SmallCtrl {
+  uint64_t full[SMALL_MAX_KB];
+  uint64_t acc_full;
+  uint32_t tmem_base;
+  int abort;
+};
+
+__device__ __forceinline__ void small_trace(const SmallParams& p, int ev) {
+  if (p.trace != nullptr && static_cast<int>(blockIdx.x) < p.trace_ctas) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    p.trace[blockIdx.x * TR_SLOTS + ev] = t;
+    if (ev == TR_START || ev == TR_END) p.trace[blockIdx.x * TR_SLOTS + (ev == TR_START ? TR_CLOCK_START : TR_CLOCK_END)] = clock64();
+  }
+}
+
+__device__ __forceinline__ bool small_wait(uint32_t bar, uint32_t parity, SmallCtrl* ctrl, const SmallParams& p) {
+  if (ptx::mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (uint32_t spin = 1;; ++spin) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    if ((spin & 31u) == 0u) {
+      if (*reinterpret_cast<volatile int*>(&ctrl->abort)) return false;
+      if (clock64() - t0 > p.wait_limit) {
+        *reinterpret_cast<volatile int*>(&ctrl->abort) = 1;
+        atomicCAS(p.status, STATUS_OK, STATUS_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+
+// One instance per activation: each is a few kilobytes of code.  (A single instance that reaches the
+// activation through a call was tried: the call's stack frame lives in local memory, cold like
+// everything else, and cost 2 us per sixteen columns.)
+template <int ACT>
+__global__ void __launch_bounds__(128, 1)
+small_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const SmallParams p) {
+  extern __shared__ uint8_t small_smem_raw[];
+  __shared__ SmallCtrl ctrl;
+  const uint32_t raw_addr = ptx::smem_u32(small_smem_raw);
+  const uint32_t ring = (raw_addr + 1023u) & ~1023u;                  // 1024-byte aligned (swizzle atoms)
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  // tile: n fastest, then m, then batch
+  const int tile = blockIdx.x;
+  const int nt = tile % p.tiles_n;
+  const int mt = (tile / p.tiles_n) % p.tiles_m;
+  const int b = tile / (p.tiles_n * p.tiles_m);
+  const int m0 = mt * BM, n0 = nt * SMALL_BN;
+
+  if (threadIdx.x == 0) {
+    ptx::prefetch_tensormap(&tmA);
+    ptx::prefetch_tensormap(&tmB);
+    small_trace(p, TR_START);
+    for (int s = 0; s < p.k_blocks; ++s) ptx::mbar_init(ptx::smem_u32(&ctrl.full[s]), 1);
+    ptx::mbar_init(ptx::smem_u32(&ctrl.acc_full), 1);
+    ctrl.abort = 0;
+    ptx::fence_mbar_init();
+    for (int kb = 0; kb < p.k_blocks; ++kb) {                          // everything at once: the ring is never reused
+      const uint32_t bar = ptx::smem_u32(&ctrl.full[kb]);
+      const uint32_t a_dst = ring + kb * SMALL_STAGE_BYTES;
+      ptx::mbar_arrive_expect_tx(bar, SMALL_STAGE_BYTES);
+      if (!(p.test_starve && kb == 0)) ptx::tma_load_3d(a_dst, &tmA, bar, kb * BK, m0, b);
+      if (p.b_kmajor) ptx::tma_load_3d(a_dst + SMALL_A_BYTES, &tmB, bar, kb * BK, n0, b);
+      else ptx::tma_load_3d(a_dst + SMALL_A_BYTES, &tmB, bar, n0, kb * BK, b);
+      if (kb == 0) small_trace(p, TR_FIRST_LOAD);
+    }
+    small_trace(p, TR_LAST_LOAD);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc<1>(ptx::smem_u32(&ctrl.tmem_base), SMALL_TMEM_COLS);
+    ptx::tmem_relinquish<1>();
+  }
+  // bias of this tile: columns n0 + lane and n0 + 32 + lane, fetched while the operands travel
+  float bias_lo = 0.0f, bias_hi = 0.0f;
+  if (p.bias != nullptr) {
+    const int c0 = n0 + lane, c1 = n0 + 32 + lane;
+    if (p.bias_bf16) {
+      const __nv_bfloat16* bp = static_cast<const __nv_bfloat16*>(p.bias);
+      if (c0 < p.N) bias_lo = __bfloat162float(bp[c0]);
+      if (c1 < p.N) bias_hi = __bfloat162float(bp[c1]);
+    } else {
+      const float* bp = static_cast<const float*>(p.bias);
+      if (c0 < p.N) bias_lo = __ldg(bp + c0);
+      if (c1 < p.N) bias_hi = __ldg(bp + c1);
+    }
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&ctrl.tmem_base);
+  if (threadIdx.x == 0) small_trace(p, TR_SETUP_DONE);
+
+  if (threadIdx.x == 0) {
+    // ---- MMA issue: k-blocks in order as they land
+    const uint32_t idesc = ptx::instr_desc_bf16(BM, SMALL_BN, !p.b_kmajor);
+    const uint32_t b_kstep = p.b_kmajor ? ((UMMA_K * 2) >> 4) : ((UMMA_K * 128) >> 4);
+    int tail_nk = (p.K - (p.k_blocks - 1) * BK + UMMA_K - 1) / UMMA_K;      // 16-wide steps of the last k-block
+    if (tail_nk > BK / UMMA_K) tail_nk = BK / UMMA_K;
+    bool ok = true;
+    for (int kb = 0; kb < p.k_blocks && ok; ++kb) {
+      if (!small_wait(ptx::smem_u32(&ctrl.full[kb]), 0, &ctrl, p)) { ok = false; break; }
+      if (kb == 0) small_trace(p, TR_FIRST_FULL);
+      ptx::tc_fence_after();
+      const uint32_t a_addr = ring + kb * SMALL_STAGE_BYTES;
+      const uint64_t a_desc = ptx::smem_desc_sw128(a_addr, 16, 8 * 128);
+      const uint64_t b_desc = ptx::smem_desc_sw128(a_addr + SMALL_A_BYTES, p.b_kmajor ? 16 : 64 * BK * 2, 8 * 128);
+      const int nk = (kb == p.k_blocks - 1) ? tail_nk : BK / UMMA_K;
+      for (int k = 0; k < nk; ++k)
+        ptx::mma_f16<1>(tmem_base, a_desc + static_cast<uint64_t>(k * ((UMMA_K * 2) >> 4)),
+                        b_desc + static_cast<uint64_t>(k * b_kstep), idesc, (kb | k) ? 1u : 0u);
+    }
+    if (ok) {
+      ptx::tc_commit<1>(ptx::smem_u32(&ctrl.acc_full));
+      small_trace(p, TR_LAST_MMA);
+    } else {
+      // abort path: let the copies in flight land (bounded) before shared memory is given up
+      for (int kb = (p.test_starve ? 1 : 0); kb < p.k_blocks; ++kb) {
+        const long long t0 = clock64();
+        while (!ptx::mbar_try_wait(ptx::smem_u32(&ctrl.full[kb]), 0))
+          if (clock64() - t0 > (1ll << 27)) break;
+      }
+      const long long t1 = clock64();
+      while (clock64() - t1 < 100000) {}
+    }
+  }
+  __syncwarp();
+
+  // ---- epilogue: all four warps
+  if (small_wait(ptx::smem_u32(&ctrl.acc_full), 0, &ctrl, p)) {
+    ptx::tc_fence_after();
+    if (threadIdx.x == 0) small_trace(p, TR_ACC_SEEN);
+    const int m = m0 + warp * 32 + lane;
+    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
+    const bool has_r = p.beta != 0.0f;
+    const size_t row_off = (static_cast<size_t>(b) * p.M + (m < p.M ? m : 0)) * p.N;
+#pragma unroll 1
+    for (int g = 0; g < SMALL_BN / 16; ++g) {
+      const int col = n0 + g * 16;
+      if (col >= p.N) break;                                 // (uniform: the tile's columns end here)
+      uint32_t v[16];
+      ptx::tmem_ld_32x32b_x16(taddr + g * 16, v);
+      uint4 r0 = make_uint4(0, 0, 0, 0), r1 = make_uint4(0, 0, 0, 0);
+      if (has_r && m < p.M) {
+        const uint4* rp = reinterpret_cast<const uint4*>(p.R + row_off + col);
+        r0 = __ldg(rp);
+        if (col + 8 < p.N) r1 = __ldg(rp + 1);
+      }
+      ptx::tmem_ld_wait();
+      const uint32_t rw[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+      uint32_t o[8];
+#pragma unroll
+      for (int j = 0; j < 16; j += 2) {
+        float u[2];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int c = g * 16 + j + e;                      // column inside the tile
+          const float bv = __shfl_sync(0xFFFFFFFFu, c < 32 ? bias_lo : bias_hi, c & 31);
+          u[e] = activate<ACT>(fmaf(p.alpha, __uint_as_float(v[j + e]), bv));
+        }
+        if (has_r) {
+          u[0] = fmaf(p.beta, __uint_as_float(rw[j >> 1] << 16), u[0]);
+          u[1] = fmaf(p.beta, __uint_as_float(rw[j >> 1] & 0xFFFF0000u), u[1]);
+        }
+        o[j >> 1] = pack_bf16x2(u[0], u[1]);
+      }
+      if (m < p.M) {
+        uint4* dp = reinterpret_cast<uint4*>(p.D + row_off + col);
+        dp[0] = make_uint4(o[0], o[1], o[2], o[3]);
+        if (col + 8 < p.N) dp[1] = make_uint4(o[4], o[5], o[6], o[7]);
+      }
+      if (threadIdx.x == 0) small_trace(p, g == 0 ? TR_FIRST_STORE : TR_LAST_STORE);
+    }
+    if (threadIdx.x == 0) small_trace(p, TR_STORES_DONE);
+  }
+
+  // ---- tear-down
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc<1>(tmem_base, SMALL_TMEM_COLS);
+  }
+  if (threadIdx.x == 0) small_trace(p, TR_END);
+}
+
+}  // namespace cg

@@ -160,10 +160,10 @@ from cg_inputs import workloads as W
 import parity_util as PU
 p = W.make(256, 256, 256, seed=5, A=("smallint", 1.0), B=("smallint", 1.0))
 dev = PU.to_device(p)
-for group in (1, 2):
+for group in (1, 2, 0):                       # 0: no plan override -- this small problem takes the latency kernel
     os.environ["CG_TEST_STARVE"] = "1"; os.environ["CG_WAIT_LIMIT_CYCLES"] = "20000000"
     bad = cg.Context(0)                       # its producer withholds one load: `full[0]` is never completed
-    bad.set_tuning(tile_n=128, cta_group=group)
+    if group: bad.set_tuning(tile_n=128, cta_group=group)
     rc = cg.cg_gemm_epilogue(bad.handle, dev["A"], dev["B"], None, None, dev["D"], 256, 256, 256, 1, 1.0, 0.0, 0)
     assert rc == cg.CG_OK, rc                 # the launch itself succeeds
     code, msg = cg.cg_last_error(bad.handle, sync=True)
@@ -172,8 +172,9 @@ for group in (1, 2):
     bad.close()
     os.environ.pop("CG_TEST_STARVE"); os.environ.pop("CG_WAIT_LIMIT_CYCLES")
     good = cg.Context(0)                      # the CUDA context is still usable and tensor memory was freed
-    good.set_tuning(tile_n=128, cta_group=group)
+    if group: good.set_tuning(tile_n=128, cta_group=group)
     d = PU.run_gpu(good, p, dev)
+    assert good.last_plan()["latency_kernel"] == (0 if group else 1)
     from oracle import ref
     r64, r16 = PU.oracle_full(ref, p)
     assert np.array_equal(d, r16)

@@ -181,6 +181,52 @@ def test_epilogue_variants(ctx, oracle, act, bias, residual):
     check(ctx, oracle, p, tile_n=512, cta_group=2)
 
 
+# ------------------------------------------------------------------ the latency kernel (small problems, no plan override)
+
+@pytest.mark.parametrize("colmajor", [False, True])
+@pytest.mark.parametrize("shape", [(128, 64, 64, 1), (1, 8, 8, 1), (127, 72, 8, 2), (129, 136, 200, 1), (200, 264, 72, 3),
+                                   (256, 256, 256, 1), (384, 512, 512, 1), (33, 40, 456, 5), (640, 200, 504, 2)],
+                         ids=lambda s: "x".join(map(str, s)))
+def test_latency_kernel_integer_operands_bit_exact(ctx, oracle, shape, colmajor):
+    M, N, K, batch = shape
+    act = W.ACT_RELU | (W.FLAG_B_COLMAJOR if colmajor else 0)
+    p = W.make(M, N, K, batch, seed=M + N + K, act=act, alpha=2.0, beta=-1.0, A=SI, B=SI, bias=SI, R=SI)
+    plan = check(ctx, oracle, p, exact=True)
+    assert plan["latency_kernel"] == 1 and plan["grid"] == batch * ((M + 127) // 128) * ((N + 63) // 64) and plan["launches"] == 1
+    assert plan["stages"] == (K + 63) // 64
+
+
+@pytest.mark.parametrize("act", ALL_ACTS)
+@pytest.mark.parametrize("bias", [None, "f32", "bf16"])
+@pytest.mark.parametrize("residual", [False, True])
+def test_latency_kernel_epilogue_variants(ctx, oracle, act, bias, residual):
+    flags = W.FLAG_BIAS_BF16 if bias == "bf16" else 0
+    p = W.make(300, 328, 264, batch=2, seed=act * 5 + (2 if residual else 0), act=act | flags, alpha=0.75,
+               beta=1.5 if residual else 0.0, A=("normal", 1.0), B=("normal", 0.1),
+               bias=None if bias is None else ("normal", 1.0), R=("normal", 1.0) if residual else None)
+    assert check(ctx, oracle, p)["latency_kernel"] == 1
+
+
+def test_latency_kernel_in_place_residual_and_limits(ctx, oracle):
+    import torch
+    p = W.make(256, 192, 320, seed=8, act=W.ACT_SILU, alpha=0.5, beta=1.0, A=("normal", 1.0), B=("normal", 0.1),
+               bias=("normal", 1.0), R=("normal", 1.0))
+    dev = PU.to_device(p)
+    dev["D"] = dev["R"]                                                   # D aliases R exactly
+    ctx.set_tuning(reset=True)
+    d = PU.run_gpu(ctx, p, dev)
+    assert ctx.last_plan()["latency_kernel"] == 1
+    r64, _ = PU.oracle_full(oracle, p)
+    assert PU.compare(d, r64)["ok"]
+    # just past each limit the persistent kernel runs instead
+    for shape in [(128, 64, 576, 1), (128, 64 * 149, 64, 1), (1024, 520, 64, 1)]:       # K > 512; more tiles than SMs; > 2^19 outputs
+        q = W.make(*shape[:3], batch=shape[3], seed=3, act=W.ACT_RELU, A=SI, B=SI, bias=SI)
+        assert check(ctx, oracle, q, exact=True)["latency_kernel"] == 0
+    # ... as with any plan override
+    q = W.make(256, 256, 256, seed=3, act=W.ACT_RELU, A=SI, B=SI, bias=SI)
+    assert check(ctx, oracle, q, exact=True, stages=2)["latency_kernel"] == 0
+
+
 def test_activation_tails(ctx, oracle):
     """Large |t| through the exponential-based activations: no NaN from exp overflow, correct limits."""
     for act in (W.ACT_SILU, W.ACT_GELU_TANH, W.ACT_GELU_ERF, W.ACT_SIGMOID, W.ACT_TANH):
