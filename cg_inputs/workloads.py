@@ -6,7 +6,7 @@ low byte = activation (0 none, 1 ReLU, 2 GELU-tanh, 3 SiLU, 4 GELU-erf, 5 sigmoi
 7 leaky ReLU with slope 0.01); bit 8 = B stored column-major
 ([batch,N,K]); bit 9 = bias is bf16 instead of fp32.  Extended entry point only: bit 10 = the bias
 is per output row (length M); bit 11 = one B shared by all batch entries; bit 12 = clamp the
-activation's result to [clamp_lo, clamp_hi].  Output dtype codes: 0 bf16, 1 fp16, 2 fp32.
+activation's result to [clamp_lo, clamp_hi]; bit 13 = A and B are float32 and multiplied as TF32.  Output dtype codes: 0 bf16, 1 fp16, 2 fp32.
 """
 from __future__ import annotations
 
@@ -25,6 +25,7 @@ FLAG_BIAS_BF16 = 1 << 9
 FLAG_BIAS_PER_ROW = 1 << 10
 FLAG_B_BROADCAST = 1 << 11
 FLAG_CLAMP = 1 << 12
+FLAG_IN_F32 = 1 << 13
 OUT_BF16, OUT_F16, OUT_F32 = 0, 1, 2
 
 
@@ -38,7 +39,7 @@ class Problem:
     alpha: float
     beta: float
     act: int                      # activation | flags
-    A: np.ndarray                 # uint16 bf16 bits [batch, M, K]
+    A: np.ndarray                 # uint16 bf16 bits [batch, M, K] (float32 with FLAG_IN_F32, also B)
     B: np.ndarray                 # uint16 bf16 bits [batch, K, N] or [batch, N, K] (column-major flag)
     bias: Optional[np.ndarray]    # float32 [N] / uint16 bf16 bits [N] / None
     R: Optional[np.ndarray]       # uint16 bf16 bits [batch, M, N] / None
@@ -53,7 +54,7 @@ class Problem:
 
     @property
     def extended(self) -> bool:
-        return bool(self.act & (FLAG_BIAS_PER_ROW | FLAG_B_BROADCAST | FLAG_CLAMP)) or self.row_scale is not None \
+        return bool(self.act & (FLAG_BIAS_PER_ROW | FLAG_B_BROADCAST | FLAG_CLAMP | FLAG_IN_F32)) or self.row_scale is not None \
             or self.col_scale is not None or self.out_dtype != OUT_BF16
 
     @property
@@ -65,7 +66,8 @@ class Problem:
         """Each operand read once, D written once."""
         out_bytes = 4 if self.out_dtype == OUT_F32 else 2
         b_entries = 1 if self.act & FLAG_B_BROADCAST else self.batch
-        b = 2 * self.batch * self.M * self.K + 2 * b_entries * self.K * self.N + out_bytes * self.batch * self.M * self.N
+        in_bytes = 4 if self.act & FLAG_IN_F32 else 2
+        b = in_bytes * (self.batch * self.M * self.K + b_entries * self.K * self.N) + out_bytes * self.batch * self.M * self.N
         for v in (self.row_scale, self.col_scale):
             if v is not None:
                 b += v.nbytes
@@ -103,8 +105,10 @@ def make(M, N, K, batch=1, seed=0, act=ACT_NONE, alpha=1.0, beta=0.0, A=("unifor
     ``col_scale``: distribution specs of fp32 vectors ("pow2" draws exact powers of two 2^-2..2^2);
     ``clamp``: (lo, hi), sets FLAG_CLAMP."""
     colmajor = bool(act & FLAG_B_COLMAJOR)
-    a = gen.tensor(seed, gen.TENSOR_A, (batch, M, K), A[0], A[1])
-    b = gen.tensor(seed, gen.TENSOR_B, (1 if act & FLAG_B_BROADCAST else batch, K, N), B[0], B[1], colmajor_last2=colmajor)
+    in_dtype = "f32" if act & FLAG_IN_F32 else "bf16"
+    a = gen.tensor(seed, gen.TENSOR_A, (batch, M, K), A[0], A[1], dtype=in_dtype)
+    b = gen.tensor(seed, gen.TENSOR_B, (1 if act & FLAG_B_BROADCAST else batch, K, N), B[0], B[1], dtype=in_dtype,
+                   colmajor_last2=colmajor)
     bias_arr = None
     if bias is not None:
         want = "bf16" if act & FLAG_BIAS_BF16 else "f32"

@@ -38,6 +38,11 @@
 //   with bias = bias[n], or bias[m] under the per-row flag; b' = b, or 0 when one B is shared by all
 //   batch entries; missing scale vectors count as 1; the output is rounded once from fp64 to bf16,
 //   fp16 or fp32 (nearest-even).  With every extension off this is the formula above, bit for bit.
+//   With the fp32-input flag A and B are fp32 and are multiplied as TF32 (the precision of the paper's
+//   square-GEMM case study: fp32 tensors, TF32 tensor-core multiply, fp32 accumulate): each operand
+//   keeps its sign, exponent and upper 10 fraction bits, the 13 low fraction bits are dropped
+//   (truncation: a tensor core fed fp32 data ignores those bits), products and sums are then exact
+//   fp64 as everywhere else.
 //   Readings: the scales multiply the product only (like alpha), never the bias; the clamp follows the
 //   activation and precedes the residual; scale vectors and per-row bias are shared by the batch.
 //
@@ -90,7 +95,7 @@ enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU_TANH = 2, ACT_SILU = 3,
 constexpr int ACT_LAST = ACT_LEAKY_RELU;
 constexpr double LEAKY_SLOPE = 0.01;
 enum { FLAG_B_COLMAJOR = 1 << 8, FLAG_BIAS_BF16 = 1 << 9, FLAG_BIAS_PER_ROW = 1 << 10, FLAG_B_BROADCAST = 1 << 11,
-       FLAG_CLAMP = 1 << 12 };
+       FLAG_CLAMP = 1 << 12, FLAG_IN_F32 = 1 << 13 };
 enum { OUT_BF16 = 0, OUT_F16 = 1, OUT_F32 = 2 };
 
 // fp64 -> fp16 bit pattern, round to nearest, ties to even, in one rounding step.
@@ -118,6 +123,15 @@ inline uint16_t f64_to_f16_rne(double v) {
   return sign | static_cast<uint16_t>(biased << 10) | frac;
 }
 
+// fp32 -> the value a TF32 multiplier sees: the 13 low fraction bits dropped.
+inline double f32_as_tf32(float f) {
+  uint32_t w;
+  std::memcpy(&w, &f, sizeof w);
+  w &= 0xFFFFE000u;
+  std::memcpy(&f, &w, sizeof f);
+  return static_cast<double>(f);
+}
+
 inline double activation(int act, double t) {
   switch (act) {
     case ACT_RELU:
@@ -140,8 +154,8 @@ inline double activation(int act, double t) {
 }
 
 struct Problem {
-  const uint16_t* A;
-  const uint16_t* B;
+  const void* A;          // bf16 bit patterns, or fp32 with in_f32
+  const void* B;
   const void* bias;
   const uint16_t* R;
   int64_t M, N, K, batch;
@@ -149,7 +163,7 @@ struct Problem {
   int act;
   bool b_colmajor, bias_bf16;
   // extended family (all off in the base entry points)
-  bool bias_per_row = false, b_broadcast = false, clamp = false;
+  bool bias_per_row = false, b_broadcast = false, clamp = false, in_f32 = false;
   const float* row_scale = nullptr;   // [M] or null
   const float* col_scale = nullptr;   // [N] or null
   double clamp_lo = 0.0, clamp_hi = 0.0;
@@ -164,11 +178,18 @@ inline double bias_at(const Problem& p, int64_t m, int64_t n) {
   return static_cast<double>(static_cast<const float*>(p.bias)[i]);
 }
 
+// Operand element i as the multiplier sees it: a bf16 value, or an fp32 value cut to TF32.
+inline double operand(const Problem& p, const void* base, int64_t i) {
+  if (p.in_f32) return f32_as_tf32(static_cast<const float*>(base)[i]);
+  return bf16_to_f64(static_cast<const uint16_t*>(base)[i]);
+}
+inline double a_at(const Problem& p, int64_t b, int64_t m, int64_t k) { return operand(p, p.A, (b * p.M + m) * p.K + k); }
+
 // B[b,k,n] through an index function: row-major [batch,K,N] or column-major [batch,N,K];
 // a shared B has a single batch entry.
 inline double b_at(const Problem& p, int64_t b, int64_t k, int64_t n) {
   const int64_t base = (p.b_broadcast ? 0 : b) * p.K * p.N;
-  return bf16_to_f64(p.b_colmajor ? p.B[base + n * p.K + k] : p.B[base + k * p.N + n]);
+  return operand(p, p.B, p.b_colmajor ? base + n * p.K + k : base + k * p.N + n);
 }
 
 inline double finish(const Problem& p, int64_t b, int64_t m, int64_t n, double s) {
@@ -197,7 +218,7 @@ void row(const Problem& p, int64_t b, int64_t m, std::vector<double>& acc, doubl
          void* out16) {
   for (int64_t n = 0; n < p.N; ++n) acc[n] = 0.0;
   for (int64_t k = 0; k < p.K; ++k) {
-    const double a = bf16_to_f64(p.A[(b * p.M + m) * p.K + k]);
+    const double a = a_at(p, b, m, k);
     for (int64_t n = 0; n < p.N; ++n) acc[n] += a * b_at(p, b, k, n);
   }
   for (int64_t n = 0; n < p.N; ++n) {
@@ -210,8 +231,8 @@ void row(const Problem& p, int64_t b, int64_t m, std::vector<double>& acc, doubl
 Problem make(const void* A, const void* B, const void* bias, const void* R, int64_t M, int64_t N,
              int64_t K, int64_t batch, double alpha, double beta, int act) {
   Problem p;
-  p.A = static_cast<const uint16_t*>(A);
-  p.B = static_cast<const uint16_t*>(B);
+  p.A = A;
+  p.B = B;
   p.bias = bias;
   p.R = static_cast<const uint16_t*>(R);
   p.M = M; p.N = N; p.K = K; p.batch = batch;
@@ -229,6 +250,7 @@ Problem make_ex(const void* A, const void* B, const void* bias, const void* R, i
   p.bias_per_row = (act & FLAG_BIAS_PER_ROW) != 0;
   p.b_broadcast = (act & FLAG_B_BROADCAST) != 0;
   p.clamp = (act & FLAG_CLAMP) != 0;
+  p.in_f32 = (act & FLAG_IN_F32) != 0;
   p.row_scale = row_scale;
   p.col_scale = col_scale;
   p.clamp_lo = clamp_lo;
@@ -288,7 +310,7 @@ int cg_ref_gemm_epilogue_points(const void* A, const void* B, const void* bias, 
     if (idx[i] < 0 || idx[i] >= batch * M * N) return 1;
     const int64_t n = idx[i] % N, bm = idx[i] / N, m = bm % M, b = bm / M;
     double s = 0.0;
-    for (int64_t k = 0; k < K; ++k) s += bf16_to_f64(p.A[(b * M + m) * K + k]) * b_at(p, b, k, n);
+    for (int64_t k = 0; k < K; ++k) s += a_at(p, b, m, k) * b_at(p, b, k, n);
     const double v = finish(p, b, m, n, s);
     if (d64) d64[i] = v;
     if (d16) d16[i] = f64_to_bf16_rne(v);
@@ -319,6 +341,7 @@ int cg_ref_gemm_epilogue_ex(const void* A, const void* B, const void* bias, cons
 
 // Helpers exposed so the pins can exercise them directly.
 uint16_t cg_ref_f64_to_f16(double v) { return f64_to_f16_rne(v); }
+double cg_ref_f32_as_tf32(float f) { return f32_as_tf32(f); }
 double cg_ref_activation(int act, double t) { return activation(act & 0xFF, t); }
 uint16_t cg_ref_f64_to_bf16(double v) { return f64_to_bf16_rne(v); }
 double cg_ref_bf16_to_f64(uint16_t h) { return bf16_to_f64(h); }

@@ -22,6 +22,7 @@ FLAG_BIAS_BF16 = 1 << 9
 FLAG_BIAS_PER_ROW = 1 << 10
 FLAG_B_BROADCAST = 1 << 11
 FLAG_CLAMP = 1 << 12
+FLAG_IN_F32 = 1 << 13
 OUT_BF16, OUT_F16, OUT_F32 = 0, 1, 2
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -72,6 +73,8 @@ def _load():
         lib.cg_ref_gemm_epilogue_ex.argtypes = [vp, vp, vp, vp, vp, i64, vp, vp, i64, i64, i64, i64, dbl, dbl, ci, vp, vp,
                                                 dbl, dbl, ci]
         lib.cg_ref_gemm_epilogue_ex.restype = ci
+        lib.cg_ref_f32_as_tf32.argtypes = [ctypes.c_float]
+        lib.cg_ref_f32_as_tf32.restype = dbl
         lib.cg_ref_f64_to_f16.argtypes = [dbl]
         lib.cg_ref_f64_to_f16.restype = ctypes.c_uint16
         lib.cg_ref_activation.argtypes = [ci, dbl]
@@ -144,12 +147,14 @@ def gemm_epilogue_points(A, B, bias, R, idx, M, N, K, batch, alpha, beta, act):
 
 def gemm_epilogue_ex(A, B, bias, R, M, N, K, batch, alpha, beta, act, row_scale=None, col_scale=None, clamp_lo=0.0,
                      clamp_hi=0.0, out_dtype=OUT_BF16, rows=None):
-    """Extended consumer family: scale vectors, per-row bias, clamp, shared B, bf16 / fp16 / fp32 output.
+    """Extended consumer family: scale vectors, per-row bias, clamp, shared B, bf16 / fp16 / fp32 output,
+    and (FLAG_IN_F32) float32 operands multiplied as TF32.
     Returns (D64, Dout) for the whole problem ([batch,M,N]) or for ``rows`` ([len(rows),N]); Dout is
     uint16 bit patterns (bf16, fp16) or float32."""
+    in_dtype = np.float32 if act & FLAG_IN_F32 else np.uint16
     for name, x, n in (("A", A, batch * M * K), ("B", B, (1 if act & FLAG_B_BROADCAST else batch) * K * N)):
-        if x.dtype != np.uint16 or not x.flags.c_contiguous or x.size != n:
-            raise TypeError(f"{name} must be a C-contiguous uint16 (bf16 bits) array of the right size")
+        if x.dtype != in_dtype or not x.flags.c_contiguous or x.size != n:
+            raise TypeError(f"{name} must be a C-contiguous {in_dtype.__name__} array of the right size")
     if bias is not None:
         want = np.uint16 if act & FLAG_BIAS_BF16 else np.float32
         if bias.dtype != want or bias.size != (M if act & FLAG_BIAS_PER_ROW else N) or not bias.flags.c_contiguous:
@@ -169,6 +174,10 @@ def gemm_epilogue_ex(A, B, bias, R, M, N, K, batch, alpha, beta, act, row_scale=
     if rc != 0:
         raise ValueError("oracle rejected the arguments")
     return d64, dout
+
+
+def f32_as_tf32(v):
+    return float(_load().cg_ref_f32_as_tf32(float(v)))
 
 
 def f64_to_f16(v):

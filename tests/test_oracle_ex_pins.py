@@ -184,3 +184,61 @@ def test_typed_outputs_are_one_rounding_of_the_fp64_result(oracle, out_dtype):
         assert np.array_equal(eout, e64.astype(np.float16).view(np.uint16))
     b64, _ = oracle.gemm_epilogue(p.A, p.B, p.bias, None, p.M, p.N, p.K, p.batch, p.alpha, 0.0, p.act)
     assert np.array_equal(b64, e64)                                                 # the dtype changes only the rounding
+
+
+# ---------------------------------------------------------------- fp32 operands multiplied as TF32
+
+def np_tf32(x):
+    """numpy's view of the same cut: clear the 13 low fraction bits of each float32."""
+    return (np.ascontiguousarray(x, dtype=np.float32).view(np.uint32) & np.uint32(0xFFFFE000)).view(np.float32)
+
+
+def test_tf32_cut_properties(oracle):
+    rng = np.random.default_rng(1)
+    x = np.concatenate([rng.normal(0, 1, 3000), rng.normal(0, 1e-30, 500), rng.normal(0, 1e30, 500),
+                        np.array([0.0, -0.0, 1.0, 1.0 + 2.0 ** -10, 1.0 + 2.0 ** -11, 2.0 - 2.0 ** -23, -(2.0 - 2.0 ** -23)])]).astype(np.float32)
+    got = np.array([oracle.f32_as_tf32(v) for v in x.tolist()])
+    assert np.array_equal(got, np_tf32(x).astype(np.float64))
+    assert np.all(np.abs(got) <= np.abs(x.astype(np.float64)))                       # towards zero
+    assert np.all(np.abs(got - x) <= np.abs(x.astype(np.float64)) * 2.0 ** -10)      # within one TF32 ulp
+    assert np.array_equal(np.array([oracle.f32_as_tf32(v) for v in got.tolist()]), got)   # idempotent
+    assert oracle.f32_as_tf32(1.0 + 2.0 ** -11) == 1.0 and oracle.f32_as_tf32(1.0 + 2.0 ** -10) == 1.0 + 2.0 ** -10
+    # every finite bf16 value has at most 7 fraction bits: TF32 keeps it whole
+    allbf = gen.bf16_bits_to_f32(np.arange(65536, dtype=np.uint16))
+    fin = allbf[np.isfinite(allbf)]
+    assert np.array_equal(np.array([oracle.f32_as_tf32(v) for v in fin.tolist()]), fin.astype(np.float64))
+
+
+def test_tf32_on_bf16_representable_values_is_the_bf16_path(oracle):
+    M, N, K, batch = 19, 24, 40, 2
+    p = W.make(M, N, K, batch, seed=14, act=W.ACT_SILU | W.FLAG_B_COLMAJOR, alpha=0.5, beta=1.0, A=("normal", 1.0),
+               B=("normal", 0.5), bias=("normal", 1.0), R=("normal", 1.0))
+    b64, b16 = oracle.gemm_epilogue(p.A, p.B, p.bias, p.R, M, N, K, batch, p.alpha, p.beta, p.act)
+    a32, b32 = gen.bf16_bits_to_f32(p.A), gen.bf16_bits_to_f32(p.B)
+    e64, e16 = oracle.gemm_epilogue_ex(a32, b32, p.bias, p.R, M, N, K, batch, p.alpha, p.beta, p.act | W.FLAG_IN_F32)
+    assert np.array_equal(b64, e64) and np.array_equal(b16, e16)
+
+
+@pytest.mark.parametrize("colmajor", [False, True])
+def test_tf32_random_fp32_against_numpy_on_cut_operands(oracle, colmajor):
+    M, N, K, batch = 17, 16, 56, 2
+    flags = W.FLAG_IN_F32 | (W.FLAG_B_COLMAJOR if colmajor else 0)
+    p = W.make(M, N, K, batch, seed=15, act=flags, alpha=1.25, A=("normal", 1.0), B=("normal", 1.0), bias=("normal", 1.0),
+               out_dtype=W.OUT_F32)
+    assert p.A.dtype == np.float32 and not np.array_equal(np_tf32(p.A), p.A)          # the cut does change these operands
+    e64, e32 = run_ex(oracle, p)
+    bm = np.swapaxes(p.B, 1, 2) if colmajor else p.B
+    want = p.alpha * np.einsum("bmk,bkn->bmn", np_tf32(p.A).astype(np.float64), np_tf32(bm).astype(np.float64)) \
+        + p.bias.astype(np.float64)[None, None, :]
+    assert np.allclose(e64, want, rtol=1e-12, atol=1e-12)
+    assert np.array_equal(e32, e64.astype(np.float32))
+    uncut = p.alpha * np.einsum("bmk,bkn->bmn", p.A.astype(np.float64), bm.astype(np.float64)) + p.bias.astype(np.float64)[None, None, :]
+    assert not np.allclose(e64, uncut, rtol=1e-6, atol=1e-6)                          # (and it matters at this scale)
+
+
+def test_tf32_small_integers_exact(oracle):
+    M, N, K = 13, 16, 64
+    p = W.make(M, N, K, seed=16, act=W.FLAG_IN_F32 | W.FLAG_B_COLMAJOR, A=SI, B=SI, out_dtype=W.OUT_F32)
+    e64, e32 = run_ex(oracle, p)
+    want = np.einsum("bmk,bnk->bmn", p.A.astype(np.int64), p.B.astype(np.int64))
+    assert np.array_equal(e64, want.astype(np.float64)) and np.array_equal(e32, want.astype(np.float32))
