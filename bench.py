@@ -358,6 +358,40 @@ def extended_sweep(ctx, p, dev, flush):
     return out
 
 
+def tf32_row(ctx, device, peaks, flush):
+    """fp32 operands multiplied as TF32 (the precision of the paper's square-GEMM case study), 8192^3 with
+    B stored [N,K], bias + SiLU, fp32 output; cuBLAS TF32 through torch.matmul alongside (GEMM alone).  The
+    peak is the measured bf16 peak times the nominal TF32 / bf16 ratio (1.1 / 2.25)."""
+    import torch
+    n = 8192
+    g = torch.Generator(device=device)
+    g.manual_seed(5)
+    A = torch.randn((1, n, n), device=device, generator=g) / 90.0
+    B = torch.randn((1, n, n), device=device, generator=g) / 90.0            # [N, K]
+    bias = torch.randn((n,), device=device, generator=g) * 0.02
+    D = torch.empty((1, n, n), device=device, dtype=torch.float32)
+    act = W.ACT_SILU | W.FLAG_B_COLMAJOR | W.FLAG_IN_F32
+    call = lambda: ctx.gemm_epilogue_ex(A, B, bias, None, D, n, n, n, 1, 1.0, 0.0, act, out_dtype=W.OUT_F32)
+    timed(call, 3, flush)
+    ts = timed(call, 10, flush)
+    ctx.check()
+    plan = ctx.last_plan()
+    old = torch.backends.cuda.matmul.allow_tf32
+    torch.backends.cuda.matmul.allow_tf32 = True
+    lib = lambda: torch.matmul(A[0], B[0].t(), out=D[0])
+    timed(lib, 3, flush)
+    tl = timed(lib, 10, flush)
+    torch.backends.cuda.matmul.allow_tf32 = old
+    flops = 2.0 * n ** 3
+    peak = peaks["bf16_tflops"] * 1.1 / 2.25
+    best = min(ts)
+    return {"workload": "8192^3, A [M,K] and B [N,K] fp32 multiplied as TF32, bias fp32, SiLU, fp32 output",
+            "us_best": best * 1e6, "us_median": float(np.median(ts)) * 1e6, "tflops_best": flops / best / 1e12,
+            "peak_tflops": peak, "peak_kind": f"bf16 burst of {peaks['source']} x 1.1/2.25 (nominal TF32 / bf16 ratio)",
+            "frac_of_peak": flops / best / 1e12 / peak, "frac_of_nominal_1100": flops / best / 1e12 / 1100.0,
+            "cublas_tf32_gemm_only_us_best": min(tl) * 1e6, "plan": plan}
+
+
 def workload_table(ctx, device, peaks, names):
     """All five workloads under the heuristic plan, each launch timed alone after an L2 flush (their
     inputs may fit in L2)."""
@@ -386,6 +420,9 @@ def workload_table(ctx, device, peaks, names):
             out["activation_sweep_4096_us_best"] = activation_sweep(ctx, p, dev, flush)
             out["extended_family_4096_us_best"] = extended_sweep(ctx, p, dev, flush)
         del dev
+    if len(names) > 1:
+        ctx.set_tuning(reset=True)
+        out["next_tf32_8192"] = tf32_row(ctx, device, peaks, flush)
     return out
 
 

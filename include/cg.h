@@ -104,6 +104,10 @@ CG_API int cg_gemm_epilogue(cg_handle_t h, const void* A, const void* B, const v
  *   CG_FLAG_BIAS_PER_ROW  bias has M entries and bias[m] is added (dtype per CG_FLAG_BIAS_BF16)
  *   CG_FLAG_B_BROADCAST   B has a single batch entry ([K,N], or [N,K] with CG_FLAG_B_COLMAJOR) used by all (b' = 0)
  *   CG_FLAG_CLAMP         clamp the activation's result to [ex->clamp_lo, ex->clamp_hi] (before the residual)
+ *   CG_FLAG_IN_F32        A and B are fp32 and are multiplied as TF32 with fp32 accumulation (the precision of the
+ *                         paper's square-GEMM case study): the tensor core drops the 13 low fraction bits of each
+ *                         operand.  B must be stored [batch,N,K] (CG_FLAG_B_COLMAJOR, else CG_ERR_UNSUPPORTED);
+ *                         K % 4 == 0 would do for the fp32 row pitch, K % 8 == 0 is still required
  * and in *ex (NULL = all off, the call then equals cg_gemm_epilogue):
  *   row_scale, col_scale  device, fp32 [M] / [N], or NULL (= 1); they scale the product like alpha, never the bias;
  *                         shared by all batch entries
@@ -111,7 +115,7 @@ CG_API int cg_gemm_epilogue(cg_handle_t h, const void* A, const void* B, const v
  *                         16-byte aligned and N % 8 == 0 as before
  * Errors as for cg_gemm_epilogue; CG_ERR_INVALID_ARG also for clamp_lo > clamp_hi or CG_FLAG_CLAMP without ex.
  */
-enum { CG_FLAG_BIAS_PER_ROW = 1 << 10, CG_FLAG_B_BROADCAST = 1 << 11, CG_FLAG_CLAMP = 1 << 12 };
+enum { CG_FLAG_BIAS_PER_ROW = 1 << 10, CG_FLAG_B_BROADCAST = 1 << 11, CG_FLAG_CLAMP = 1 << 12, CG_FLAG_IN_F32 = 1 << 13 };
 enum { CG_OUT_BF16 = 0, CG_OUT_F16 = 1, CG_OUT_F32 = 2 };
 typedef struct cg_epilogue_ex {
   const float* row_scale;

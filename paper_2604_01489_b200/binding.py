@@ -20,6 +20,7 @@ CG_FLAG_BIAS_BF16 = 1 << 9
 CG_FLAG_BIAS_PER_ROW = 1 << 10
 CG_FLAG_B_BROADCAST = 1 << 11
 CG_FLAG_CLAMP = 1 << 12
+CG_FLAG_IN_F32 = 1 << 13
 CG_OUT_BF16, CG_OUT_F16, CG_OUT_F32 = 0, 1, 2
 
 STATUS_NAMES = {0: "CG_OK", 1: "CG_ERR_INVALID_ARG", 2: "CG_ERR_UNSUPPORTED", 3: "CG_ERR_ARCH", 4: "CG_ERR_CUDA",

@@ -209,10 +209,11 @@ size_t partial_need(long long split_units, int bn, int cgn) {
   return static_cast<size_t>(2) * split_units * cgn * BM * bn * sizeof(float);
 }
 
-int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, bool has_r, Plan* pl, bool r_own_only = false) {
+int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, bool has_r, Plan* pl, bool r_own_only = false,
+              int bk_elems = BK) {
   const cg_tuning_t& t = h->tuning;
   const int sms = (t.max_ctas > 0 && t.max_ctas < h->num_sms) ? t.max_ctas : h->num_sms;
-  const int k_blocks = ceil_div(K, BK);
+  const int k_blocks = ceil_div(K, bk_elems);
   auto tiles = [&](int bm, int bn) -> long long {
     return static_cast<long long>(batch) * ceil_div(M, bm) * ceil_div(N, bn);
   };
@@ -426,7 +427,7 @@ int launch_small(cg_context* h, const void* A, const void* B, const void* bias, 
 int launch(cg_context* h, const void* A, const void* B, const void* bias, const void* R, void* D, int M, int N, int K,
            int batch, float alpha, float beta, int act, cudaStream_t stream, const cg_epilogue_ex_t* ex = nullptr) {
   const bool b_kmajor = (act & CG_FLAG_B_COLMAJOR) != 0;
-  const bool ext_in_use = (act & (CG_FLAG_BIAS_PER_ROW | CG_FLAG_B_BROADCAST | CG_FLAG_CLAMP)) != 0 ||
+  const bool ext_in_use = (act & (CG_FLAG_BIAS_PER_ROW | CG_FLAG_B_BROADCAST | CG_FLAG_CLAMP | CG_FLAG_IN_F32)) != 0 ||
                           (ex && (ex->row_scale || ex->col_scale || ex->out_dtype != CG_OUT_BF16));
   if (!ext_in_use) {
     const int rs = launch_small(h, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, stream);
@@ -436,15 +437,18 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   const bool b_broadcast = (act & CG_FLAG_B_BROADCAST) != 0;
   Plan pl;
   // (an fp32 chunk leaves through the staging buffer twice: the residual cannot land there)
-  int rc = make_plan(h, M, N, K, batch, b_kmajor, beta != 0.0f, &pl, out_dtype == CG_OUT_F32);
+  const bool tf32 = (act & CG_FLAG_IN_F32) != 0;
+  const int bk_elems = tf32 ? BK / 2 : BK;
+  const int in_dtype = tf32 ? CG_OUT_F32 : CG_OUT_BF16;           // (element type code of A and B)
+  int rc = make_plan(h, M, N, K, batch, b_kmajor, beta != 0.0f, &pl, out_dtype == CG_OUT_F32, bk_elems);
   if (rc != CG_OK) return rc;
   KernelEntry e;
   lookup(pl.bn, pl.cg, b_kmajor, &e);
 
   CUtensorMap tmA, tmB, tmD, tmR;
-  if ((rc = make_map(h, &tmA, A, K, M, batch, BK, BM)) != CG_OK) return rc;
+  if ((rc = make_map(h, &tmA, A, K, M, batch, bk_elems, BM, in_dtype)) != CG_OK) return rc;
   const int b_entries = b_broadcast ? 1 : batch;
-  if (b_kmajor) rc = make_map(h, &tmB, B, K, N, b_entries, BK, e.sub_cols);
+  if (b_kmajor) rc = make_map(h, &tmB, B, K, N, b_entries, bk_elems, e.sub_cols, in_dtype);
   else rc = make_map(h, &tmB, B, N, K, b_entries, 64, BK);
   if (rc != CG_OK) return rc;
   if ((rc = make_map(h, &tmD, D, N, M, batch, out_dtype == CG_OUT_F32 ? 32 : EPI_COLS, 32, out_dtype)) != CG_OK) return rc;
@@ -480,13 +484,14 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   p.b_broadcast = b_broadcast ? 1 : 0;
   p.clamp = (act & CG_FLAG_CLAMP) ? 1 : 0;
   p.out_dtype = out_dtype;
+  p.tf32 = tf32 ? 1 : 0;
   if (ex) {
     p.clamp_lo = ex->clamp_lo;
     p.clamp_hi = ex->clamp_hi;
     p.row_scale = ex->row_scale;
     p.col_scale = ex->col_scale;
   }
-  p.ext = (p.bias_per_row || p.clamp || out_dtype != CG_OUT_BF16 || p.row_scale || p.col_scale) ? 1 : 0;
+  p.ext = (p.bias_per_row || p.clamp || out_dtype != CG_OUT_BF16 || p.row_scale || p.col_scale) ? 1 : 0;   // (epilogue only)
   p.R = (beta != 0.0f) ? static_cast<const __nv_bfloat16*>(R) : nullptr;
   p.partials = h->partials;
   p.tickets = h->tickets;
@@ -603,8 +608,11 @@ int cg_gemm_epilogue_ex(cg_handle_t h, const void* A, const void* B, const void*
                         int N, int K, int batch, float alpha, float beta, int act, const cg_epilogue_ex_t* ex, void* stream) {
   if (!h) return CG_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lock(h->mu);
-  int rc = validate(h, A, B, bias, R, D, M, N, K, batch, beta, act, CG_FLAG_BIAS_PER_ROW | CG_FLAG_B_BROADCAST | CG_FLAG_CLAMP);
+  int rc = validate(h, A, B, bias, R, D, M, N, K, batch, beta, act,
+                    CG_FLAG_BIAS_PER_ROW | CG_FLAG_B_BROADCAST | CG_FLAG_CLAMP | CG_FLAG_IN_F32);
   if (rc != CG_OK) return rc;
+  if ((act & CG_FLAG_IN_F32) && !(act & CG_FLAG_B_COLMAJOR))
+    return fail(h, CG_ERR_UNSUPPORTED, "fp32 operands need B stored [batch,N,K] (CG_FLAG_B_COLMAJOR)");
   if ((rc = check_alignment(h, A, B, (act & CG_FLAG_BIAS_PER_ROW) ? nullptr : bias, R, D, beta, act)) != CG_OK) return rc;
   if (ex) {
     if (ex->out_dtype < CG_OUT_BF16 || ex->out_dtype > CG_OUT_F32) return fail(h, CG_ERR_INVALID_ARG, "unknown output dtype %d", ex->out_dtype);

@@ -48,6 +48,8 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include <type_traits>
+
 #include "cg_ptx.cuh"
 
 namespace cg {
@@ -93,6 +95,8 @@ struct KernelParams {
   int b_broadcast;        // one B shared by all batch entries
   int clamp;              // clamp the activation's result to [clamp_lo, clamp_hi]
   int out_dtype;          // OUT_BF16 / OUT_F16 / OUT_F32
+  int tf32;               // A and B are fp32 and multiplied as TF32: a k-block is 32 elements (still 128 bytes),
+                          // one MMA covers 8 of them; B is K-major
   float clamp_lo, clamp_hi;
   const float* row_scale; // fp32 [M] or NULL: multiplies alpha for row m
   const float* col_scale; // fp32 [N] or NULL: multiplies alpha for column n
@@ -137,6 +141,7 @@ struct Cfg {
   }
   static constexpr int TMEM_COLS = ACC_BUFS * BN <= 32 ? 32 : (ACC_BUFS * BN <= 64 ? 64 : (ACC_BUFS * BN <= 128 ? 128 : (ACC_BUFS * BN <= 256 ? 256 : 512)));
   static constexpr uint32_t IDESC = ptx::instr_desc_bf16(BM * CG, MMA_N, !B_KMAJOR);
+  static constexpr uint32_t IDESC_TF32 = ptx::instr_desc_tf32(BM * CG, MMA_N);
   __host__ __device__ static constexpr int layout_bytes(int stages, bool with_r) {
     return stages * STAGE_BYTES + FIXED_BYTES + (with_r ? R_BYTES : 0);
   }
@@ -394,7 +399,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     const uint32_t bar = ptx::smem_u32(&ctrl->full[stage]);
     const uint32_t a_dst = ring_addr + stage * C::STAGE_BYTES;
     const uint32_t b_dst = a_dst + C::A_BYTES;
-    const int k0 = kb * BK;
+    const int k0 = kb * (p.tf32 ? BK / 2 : BK);        // element coordinate: 128 bytes of K per block either way
     ptx::mbar_arrive_expect_tx(bar, C::STAGE_BYTES);
     if (!withhold_a) ptx::tma_load_3d(a_dst, &tmA, bar, k0, m0, b);     // (withheld only by the starvation test hook)
 #pragma unroll
@@ -467,7 +472,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           if (!wait_bar(empty0 + stage * 8, phase ^ 1u, ctrl, p)) { ok = false; break; }
           const uint32_t a_dst = ring_addr + stage * C::STAGE_BYTES;
           const uint32_t b_dst = a_dst + C::A_BYTES;
-          const int k0 = kb * BK;
+          const int k0 = kb * (p.tf32 ? BK / 2 : BK);
           if constexpr (CG == 1) {
             issue_loads(stage, kb, m0, n0, b, bb, p.test_starve && issued == 0);
           } else {
@@ -522,7 +527,10 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     // ================================================================ MMA issuer
     // One thread feeds the tensor pipe, so its instruction count per k-block is what bounds
     // small tiles: descriptor words are precomputed and only their low (address) half moves.
-    if (lane == 0 && (CG == 1 || cta_rank == 0)) {
+    // (the role is instantiated twice, for bf16 and for TF32 operands: the choice of MMA instruction is
+    // made once, outside the loops this thread lives in)
+    auto mma_role = [&](auto tf32_tag) {
+      constexpr bool TF32 = decltype(tf32_tag)::value;
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
@@ -544,8 +552,12 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       const uint32_t empty0 = ptx::smem_u32(&ctrl->empty[0]);
       const uint32_t empty0_peer = (CG == 2) ? ptx::mapa(empty0, 1) : 0u;
       const int last_kb = p.k_blocks - 1;
-      int tail_nk = (p.K - last_kb * BK + UMMA_K - 1) / UMMA_K;           // 16-wide steps of the last k-block
+      constexpr int bk_el = TF32 ? BK / 2 : BK, mma_k_el = TF32 ? UMMA_K / 2 : UMMA_K;   // elements per k-block / per MMA
+      int tail_nk = (p.K - last_kb * bk_el + mma_k_el - 1) / mma_k_el;    // 32-byte steps of the last k-block
       if (tail_nk > BK / UMMA_K) tail_nk = BK / UMMA_K;
+      auto mma = [&](uint32_t d, uint64_t a, uint64_t b, uint32_t acc_in) {
+        if constexpr (TF32) ptx::mma_tf32<CG>(d, a, b, C::IDESC_TF32, acc_in); else ptx::mma_f16<CG>(d, a, b, C::IDESC, acc_in);
+      };
       auto desc = [&](uint32_t lo) -> uint64_t { return (static_cast<uint64_t>(desc_hi) << 32) | lo; };
       while (ok && wi.next(s)) {
         if (!wait_bar(ptx::smem_u32(&ctrl->acc_empty[acc]), acc_phase ^ 1u, ctrl, p)) { ok = false; break; }
@@ -563,14 +575,14 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             for (int k = 0; k < BK / UMMA_K; ++k)
 #pragma unroll
               for (int h = 0; h < C::NSUB; ++h)
-                ptx::mma_f16<CG>(d_tmem + h * C::MMA_N, desc(a_lo + k * A_KSTEP), desc(b_lo + k * B_KSTEP + h * SUB_STEP),
-                                 C::IDESC, k == 0 ? accumulate : 1u);
+                mma(d_tmem + h * C::MMA_N, desc(a_lo + k * A_KSTEP), desc(b_lo + k * B_KSTEP + h * SUB_STEP),
+                    k == 0 ? accumulate : 1u);
           } else {
             for (int k = 0; k < tail_nk; ++k)     // K tail: skip 16-wide steps that are all padding
 #pragma unroll
               for (int h = 0; h < C::NSUB; ++h)
-                ptx::mma_f16<CG>(d_tmem + h * C::MMA_N, desc(a_lo + k * A_KSTEP), desc(b_lo + k * B_KSTEP + h * SUB_STEP),
-                                 C::IDESC, (k > 0) ? 1u : accumulate);
+                mma(d_tmem + h * C::MMA_N, desc(a_lo + k * A_KSTEP), desc(b_lo + k * B_KSTEP + h * SUB_STEP),
+                    (k > 0) ? 1u : accumulate);
           }
           accumulate = 1u;
           ptx::tc_commit<CG>(empty0 + stage * 8);
@@ -591,6 +603,9 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         while (!ptx::mbar_try_wait(ptx::smem_u32(&ctrl->drain), 0))
           if (clock64() - t0 > (1ll << 27)) break;
       }
+    };
+    if (lane == 0 && (CG == 1 || cta_rank == 0)) {
+      if (p.tf32) mma_role(std::true_type{}); else mma_role(std::false_type{});
     }
     __syncwarp();
     if (CG == 1 && p.cluster_split > 1) {

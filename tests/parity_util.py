@@ -15,6 +15,8 @@ def to_device(p, device="cuda:0"):
     import torch
 
     def bf16(x):
+        if x is not None and x.dtype == np.float32:          # fp32 operands (multiplied as TF32) travel as they are
+            return torch.from_numpy(x).to(device)
         return None if x is None else torch.from_numpy(x.view(np.int16)).to(device).view(torch.bfloat16)
 
     bias = None
