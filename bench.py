@@ -392,6 +392,36 @@ def tf32_row(ctx, device, peaks, flush):
             "cublas_tf32_gemm_only_us_best": min(tl) * 1e6, "plan": plan}
 
 
+def diag_rows(ctx, device, peaks, flush):
+    """C = diag(d) @ B at 8192 x 8192, fp32 and bf16: achieved bytes/s (B read once, C written once) against the
+    measured copy bandwidth; PyTorch's broadcast multiply and the dense product with a materialised
+    diagonal matrix (what the structure saves) alongside."""
+    import torch
+    n = 8192
+    d = torch.rand(n, device=device) + 0.5
+    out = {}
+    for label, dt, code, esize in (("f32", torch.float32, W.OUT_F32, 4), ("bf16", torch.bfloat16, W.OUT_BF16, 2)):
+        B = torch.randn(n, n, device=device).to(dt)
+        C = torch.empty_like(B)
+        call = lambda: ctx.diag_matmul(d, B, C, n, n, code)
+        timed(call, 3, flush)
+        best = min(timed(call, 10, flush))
+        ctx.check()
+        nbytes = 2 * n * n * esize + 4 * n
+        eager = lambda: torch.mul(d[:, None].to(dt), B, out=C)
+        timed(eager, 2, flush)
+        t_eager = min(timed(eager, 10, flush))
+        dm = torch.diag(d).to(dt)
+        dense = lambda: torch.matmul(dm, B, out=C)
+        timed(dense, 2, flush)
+        t_dense = min(timed(dense, 5, flush))
+        out[label] = {"us_best": best * 1e6, "gbs": nbytes / best / 1e9, "frac_hbm_of_measured": nbytes / best / 1e9 / peaks["hbm_gbs"],
+                      "algorithmic_bytes": nbytes, "torch_broadcast_mul_us_best": t_eager * 1e6,
+                      "torch_dense_matmul_with_diag_us_best": t_dense * 1e6}
+        del B, C, dm
+    return out
+
+
 def workload_table(ctx, device, peaks, names):
     """All five workloads under the heuristic plan, each launch timed alone after an L2 flush (their
     inputs may fit in L2)."""
@@ -423,6 +453,7 @@ def workload_table(ctx, device, peaks, names):
     if len(names) > 1:
         ctx.set_tuning(reset=True)
         out["next_tf32_8192"] = tf32_row(ctx, device, peaks, flush)
+        out["next_diag_matmul_8192"] = diag_rows(ctx, device, peaks, flush)
     return out
 
 

@@ -128,6 +128,20 @@ CG_API int cg_gemm_epilogue_ex(cg_handle_t h, const void* A, const void* B, cons
                                const cg_epilogue_ex_t* ex, void* stream);
 
 /*
+ * Structured matmul C = diag(d) * B, i.e. C[i,j] = d[i] * B[i,j]: the paper's example of a product whose
+ * structure a dense vendor GEMM ignores (its results section singles out the diagonal case); here it is one
+ * bandwidth-bound pass over B instead of 2*M*M*N flops.
+ *
+ *   d      device, fp32 [M]
+ *   B, C   device, [M,N] row-major, dense, 16-byte aligned, bf16 (dtype = CG_OUT_BF16, N % 8 == 0) or
+ *          fp32 (CG_OUT_F32, N % 4 == 0); C may alias B exactly
+ * The product is formed in fp32 and rounded once to C's type (nearest even).  Asynchronous on `stream`.
+ * CG_ERR_INVALID_ARG for NULL pointers, sizes < 1 or another dtype; CG_ERR_UNSUPPORTED for the
+ * alignment rules; nothing is enqueued on error.
+ */
+CG_API int cg_diag_matmul(cg_handle_t h, const float* d, const void* B, void* C, long long M, int N, int dtype, void* stream);
+
+/*
  * Same operation with HOST buffers (same shapes, dtypes and layouts as above, in host memory;
  * pinned memory makes the copies asynchronous and faster).  Copies the operands to device
  * staging buffers owned by the handle (grown on demand and kept), runs the kernel, copies D

@@ -339,6 +339,25 @@ int cg_ref_gemm_epilogue_ex(const void* A, const void* B, const void* bias, cons
   return 0;
 }
 
+// Structured matmul C = diag(d) * B: C[i,j] = d[i] * B[i,j] in fp64, rounded once to C's type.
+// (The paper's results single out the diagonal case as structure a dense GEMM ignores; the definition is
+// the matrix product with A = diag(d) written out.)  B, C: bf16 bits (out_dtype 0) or fp32 (2); d fp32.
+int cg_ref_diag_matmul(const float* d, const void* B, double* c64, void* cout, int64_t M, int64_t N, int out_dtype) {
+  if (!d || !B || M < 1 || N < 1 || (out_dtype != OUT_BF16 && out_dtype != OUT_F32)) return 1;
+  for (int64_t i = 0; i < M; ++i)
+    for (int64_t j = 0; j < N; ++j) {
+      const double b = out_dtype == OUT_F32 ? static_cast<double>(static_cast<const float*>(B)[i * N + j])
+                                            : bf16_to_f64(static_cast<const uint16_t*>(B)[i * N + j]);
+      const double v = static_cast<double>(d[i]) * b;
+      if (c64) c64[i * N + j] = v;
+      if (cout) {
+        if (out_dtype == OUT_F32) static_cast<float*>(cout)[i * N + j] = static_cast<float>(v);
+        else static_cast<uint16_t*>(cout)[i * N + j] = f64_to_bf16_rne(v);
+      }
+    }
+  return 0;
+}
+
 // Helpers exposed so the pins can exercise them directly.
 uint16_t cg_ref_f64_to_f16(double v) { return f64_to_f16_rne(v); }
 double cg_ref_f32_as_tf32(float f) { return f32_as_tf32(f); }

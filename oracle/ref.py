@@ -73,6 +73,8 @@ def _load():
         lib.cg_ref_gemm_epilogue_ex.argtypes = [vp, vp, vp, vp, vp, i64, vp, vp, i64, i64, i64, i64, dbl, dbl, ci, vp, vp,
                                                 dbl, dbl, ci]
         lib.cg_ref_gemm_epilogue_ex.restype = ci
+        lib.cg_ref_diag_matmul.argtypes = [vp, vp, vp, vp, i64, i64, ci]
+        lib.cg_ref_diag_matmul.restype = ci
         lib.cg_ref_f32_as_tf32.argtypes = [ctypes.c_float]
         lib.cg_ref_f32_as_tf32.restype = dbl
         lib.cg_ref_f64_to_f16.argtypes = [dbl]
@@ -174,6 +176,20 @@ def gemm_epilogue_ex(A, B, bias, R, M, N, K, batch, alpha, beta, act, row_scale=
     if rc != 0:
         raise ValueError("oracle rejected the arguments")
     return d64, dout
+
+
+def diag_matmul(d, B, out_dtype=OUT_BF16):
+    """C = diag(d) @ B.  d float32 [M]; B [M,N] uint16 bf16 bits (OUT_BF16) or float32 (OUT_F32).
+    Returns (C64, C in B's type)."""
+    want = np.float32 if out_dtype == OUT_F32 else np.uint16
+    if d.dtype != np.float32 or B.dtype != want or B.ndim != 2 or d.size != B.shape[0] or not B.flags.c_contiguous:
+        raise TypeError("d must be float32 [M] and B a C-contiguous [M,N] array of the stated type")
+    c64 = np.empty(B.shape, dtype=np.float64)
+    cout = np.empty(B.shape, dtype=want)
+    rc = _load().cg_ref_diag_matmul(_ptr(np.ascontiguousarray(d)), _ptr(B), _ptr(c64), _ptr(cout), B.shape[0], B.shape[1], int(out_dtype))
+    if rc != 0:
+        raise ValueError("oracle rejected the arguments")
+    return c64, cout
 
 
 def f32_as_tf32(v):

@@ -26,7 +26,7 @@ CG_OUT_BF16, CG_OUT_F16, CG_OUT_F32 = 0, 1, 2
 STATUS_NAMES = {0: "CG_OK", 1: "CG_ERR_INVALID_ARG", 2: "CG_ERR_UNSUPPORTED", 3: "CG_ERR_ARCH", 4: "CG_ERR_CUDA",
                 5: "CG_ERR_WORKSPACE", 6: "CG_ERR_TIMEOUT"}
 
-EXPORTS = ["cg_create", "cg_gemm_epilogue", "cg_gemm_epilogue_ex", "cg_gemm_epilogue_host", "cg_set_tuning", "cg_set_trace", "cg_get_last_plan",
+EXPORTS = ["cg_create", "cg_diag_matmul", "cg_gemm_epilogue", "cg_gemm_epilogue_ex", "cg_gemm_epilogue_host", "cg_set_tuning", "cg_set_trace", "cg_get_last_plan",
            "cg_last_error", "cg_gemm_epilogue_noalloc", "cg_destroy"]
 
 
@@ -77,6 +77,7 @@ def load() -> ctypes.CDLL:
     lib.cg_gemm_epilogue.argtypes = gemm_args
     lib.cg_gemm_epilogue_host.argtypes = gemm_args
     lib.cg_gemm_epilogue_ex.argtypes = gemm_args[:-1] + [ctypes.POINTER(cg_epilogue_ex_t), vp]
+    lib.cg_diag_matmul.argtypes = [vp, vp, vp, vp, ctypes.c_longlong, ci, ci, vp]
     lib.cg_set_tuning.argtypes = [vp, ctypes.POINTER(cg_tuning_t)]
     lib.cg_set_trace.argtypes = [vp, vp, ci]
     lib.cg_get_last_plan.argtypes = [vp, ctypes.POINTER(cg_plan_info_t)]
@@ -153,6 +154,11 @@ def cg_gemm_epilogue_ex(h, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, r
                                       _stream_ptr(stream))
 
 
+def cg_diag_matmul(h, d, B, C, M, N, dtype=CG_OUT_BF16, stream=None) -> int:
+    """C = diag(d) @ B: d fp32 [M]; B, C [M,N] bf16 (dtype CG_OUT_BF16) or fp32 (CG_OUT_F32)."""
+    return load().cg_diag_matmul(h, _dev_ptr(d), _dev_ptr(B), _dev_ptr(C), int(M), int(N), int(dtype), _stream_ptr(stream))
+
+
 def cg_gemm_epilogue_host(h, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, stream=None) -> int:
     return load().cg_gemm_epilogue_host(h, _host_ptr(A), _host_ptr(B), _host_ptr(bias), _host_ptr(R), _host_ptr(D),
                                         int(M), int(N), int(K), int(batch), float(alpha), float(beta), int(act),
@@ -214,6 +220,11 @@ class Context:
 
     def gemm_epilogue_ex(self, A, B, bias, R, D, M, N, K, batch=1, alpha=1.0, beta=0.0, act=CG_ACT_NONE, stream=None, **ex):
         rc = cg_gemm_epilogue_ex(self.handle, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, stream=stream, **ex)
+        if rc != CG_OK:
+            raise CgError(rc, cg_last_error(self.handle)[1])
+
+    def diag_matmul(self, d, B, C, M, N, dtype=CG_OUT_BF16, stream=None):
+        rc = cg_diag_matmul(self.handle, d, B, C, M, N, dtype, stream)
         if rc != CG_OK:
             raise CgError(rc, cg_last_error(self.handle)[1])
 

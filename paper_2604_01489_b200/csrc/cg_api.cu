@@ -15,6 +15,7 @@
 
 #include "cg_kernel.cuh"
 #include "cg_small.cuh"
+#include "cg_diag.cuh"
 
 namespace {
 
@@ -623,6 +624,33 @@ int cg_gemm_epilogue_ex(cg_handle_t h, const void* A, const void* B, const void*
     return fail(h, CG_ERR_INVALID_ARG, "CG_FLAG_CLAMP needs the bounds of a cg_epilogue_ex_t");
   }
   return launch(h, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, static_cast<cudaStream_t>(stream), ex);
+}
+
+int cg_diag_matmul(cg_handle_t h, const float* d, const void* B, void* C, long long M, int N, int dtype, void* stream) {
+  if (!h) return CG_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(h->mu);
+  if (!d || !B || !C || M < 1 || N < 1) return fail(h, CG_ERR_INVALID_ARG, "d, B, C must not be NULL and M, N must be >= 1");
+  if (dtype != CG_OUT_BF16 && dtype != CG_OUT_F32) return fail(h, CG_ERR_INVALID_ARG, "dtype must be CG_OUT_BF16 or CG_OUT_F32");
+  const int per_vec = dtype == CG_OUT_F32 ? 4 : 8;
+  if (N % per_vec != 0 || ((reinterpret_cast<uintptr_t>(B) | reinterpret_cast<uintptr_t>(C)) & 15) || (reinterpret_cast<uintptr_t>(d) & 3))
+    return fail(h, CG_ERR_UNSUPPORTED, "rows must be whole 16-byte vectors (N %% %d == 0) and B, C 16-byte aligned", per_vec);
+  const int vec_per_row = N / per_vec;
+  const unsigned gx = static_cast<unsigned>(ceil_div(vec_per_row, DIAG_THREADS));
+  // enough row groups in flight to fill the machine several times over; each strides over the rest
+  long long groups = (M + DIAG_ROWS - 1) / DIAG_ROWS;
+  long long gy = (static_cast<long long>(h->num_sms) * 16 + gx - 1) / gx;
+  if (gy > groups) gy = groups;
+  if (gy > 65535) gy = 65535;
+  const dim3 grid(gx, static_cast<unsigned>(gy), 1);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (dtype == CG_OUT_F32)
+    diag_matmul_kernel<true><<<grid, DIAG_THREADS, 0, st>>>(d, static_cast<const uint4*>(B), static_cast<uint4*>(C), M, vec_per_row);
+  else
+    diag_matmul_kernel<false><<<grid, DIAG_THREADS, 0, st>>>(d, static_cast<const uint4*>(B), static_cast<uint4*>(C), M, vec_per_row);
+  CG_CUDA(h, cudaGetLastError());
+  h->last_status = CG_OK;
+  h->last_msg[0] = 0;
+  return CG_OK;
 }
 
 int cg_gemm_epilogue_host(cg_handle_t h, const void* A, const void* B, const void* bias, const void* R, void* D, int M,

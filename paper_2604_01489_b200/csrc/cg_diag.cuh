@@ -1,0 +1,55 @@
+// Structured matmul: C = diag(d) * B, i.e. C[i,j] = d[i] * B[i,j] -- the product a dense GEMM would spend
+// 2*M*M*N flops on is one pass over B.  Bandwidth-bound: every thread moves 16-byte vectors, four rows
+// in flight per thread, the row's scale broadcast from cache.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+namespace cg {
+
+constexpr int DIAG_THREADS = 256;
+constexpr int DIAG_ROWS = 4;          // rows a thread keeps in flight
+
+template <bool F32>
+__device__ __forceinline__ uint4 diag_scale_vec(uint4 v, float d) {
+  if constexpr (F32) {
+    v.x = __float_as_uint(__uint_as_float(v.x) * d);
+    v.y = __float_as_uint(__uint_as_float(v.y) * d);
+    v.z = __float_as_uint(__uint_as_float(v.z) * d);
+    v.w = __float_as_uint(__uint_as_float(v.w) * d);
+  } else {
+    uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float lo = __uint_as_float(w[i] << 16) * d, hi = __uint_as_float(w[i] & 0xFFFF0000u) * d;
+      __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+      w[i] = *reinterpret_cast<uint32_t*>(&h);
+    }
+    v = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+  return v;
+}
+
+// grid.x covers the 16-byte vectors of a row, grid.y strides over groups of DIAG_ROWS rows.
+template <bool F32>
+__global__ void __launch_bounds__(DIAG_THREADS) diag_matmul_kernel(const float* __restrict__ d, const uint4* __restrict__ B,
+                                                                  uint4* __restrict__ C, long long rows, int vec_per_row) {
+  const int v = blockIdx.x * DIAG_THREADS + threadIdx.x;
+  if (v >= vec_per_row) return;
+  for (long long r0 = static_cast<long long>(blockIdx.y) * DIAG_ROWS; r0 < rows; r0 += static_cast<long long>(gridDim.y) * DIAG_ROWS) {
+    uint4 x[DIAG_ROWS];
+    float s[DIAG_ROWS];
+#pragma unroll
+    for (int i = 0; i < DIAG_ROWS; ++i)
+      if (r0 + i < rows) {
+        x[i] = __ldcs(B + (r0 + i) * vec_per_row + v);       // streamed: read once
+        s[i] = __ldg(d + r0 + i);
+      }
+#pragma unroll
+    for (int i = 0; i < DIAG_ROWS; ++i)
+      if (r0 + i < rows) __stcs(C + (r0 + i) * vec_per_row + v, diag_scale_vec<F32>(x[i], s[i]));
+  }
+}
+
+}  // namespace cg
