@@ -577,6 +577,18 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_row(args):
+    """One of the rows beyond the five workloads, alone (TF32 operands, diagonal matmul)."""
+    import torch
+    import paper_2604_01489_b200 as cg
+    torch.cuda.set_device(0)
+    device = torch.device("cuda", 0)
+    ctx = cg.Context(0)
+    flush = L2Flush(device)
+    row = tf32_row(ctx, device, load_peaks(), flush) if args.row == "tf32" else diag_rows(ctx, device, load_peaks(), flush)
+    print(json.dumps({"row": args.row, "result": row}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -587,10 +599,14 @@ def main():
     ap.add_argument("--no-table", action="store_true", help="skip the five-workload table")
     for flag in ("tile-n", "cta-group", "num-units", "dp-units", "stages", "group-m", "max-ctas"):
         ap.add_argument(f"--{flag}", type=int, default=0, help="plan override for ablations (0 = heuristic)")
+    ap.add_argument("--row", choices=["tf32", "diag"], default=None,
+                    help="only that row of the 'next' part of the table (a few launches; for profiler runs)")
     ap.add_argument("--kernel-only", action="store_true",
                     help="only the device-timed region (for profiler runs): no e2e, no CPU baseline, no table")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.row:
+        run_row(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

@@ -43,6 +43,10 @@
 //   keeps its sign, exponent and upper 10 fraction bits, the 13 low fraction bits are dropped
 //   (truncation: a tensor core fed fp32 data ignores those bits), products and sums are then exact
 //   fp64 as everywhere else.
+//   Fused row reduction (the Level-2 prompt: "Fuse reduction epilogue ...", consumers "sum/mean/max/min",
+//   "logsumexp"): next to D, or instead of it, one value per output row (b, m) over its N columns of the
+//   UNROUNDED v -- the reduction consumes the producer's values before they are rounded for storage:
+//   sum_n v, max_n v, or log(sum_n exp(v)) computed as mx + log(sum_n exp(v - mx)) with mx = max_n v.
 //   Readings: the scales multiply the product only (like alpha), never the bias; the clamp follows the
 //   activation and precedes the residual; scale vectors and per-row bias are shared by the batch.
 //
@@ -97,6 +101,7 @@ constexpr double LEAKY_SLOPE = 0.01;
 enum { FLAG_B_COLMAJOR = 1 << 8, FLAG_BIAS_BF16 = 1 << 9, FLAG_BIAS_PER_ROW = 1 << 10, FLAG_B_BROADCAST = 1 << 11,
        FLAG_CLAMP = 1 << 12, FLAG_IN_F32 = 1 << 13 };
 enum { OUT_BF16 = 0, OUT_F16 = 1, OUT_F32 = 2 };
+enum { REDUCE_NONE = 0, REDUCE_SUM = 1, REDUCE_MAX = 2, REDUCE_LOGSUMEXP = 3 };
 
 // fp64 -> fp16 bit pattern, round to nearest, ties to even, in one rounding step.
 // fp16: 1 sign, 5 exponent (bias 15), 10 fraction bits; subnormals below 2^-14; largest finite 65504.
@@ -215,7 +220,7 @@ inline void put(const Problem& p, void* out, int64_t i, double v) {
 }
 
 void row(const Problem& p, int64_t b, int64_t m, std::vector<double>& acc, double* out64,
-         void* out16) {
+         void* out16, int reduce_op = REDUCE_NONE, double* reduced = nullptr) {
   for (int64_t n = 0; n < p.N; ++n) acc[n] = 0.0;
   for (int64_t k = 0; k < p.K; ++k) {
     const double a = a_at(p, b, m, k);
@@ -225,6 +230,21 @@ void row(const Problem& p, int64_t b, int64_t m, std::vector<double>& acc, doubl
     const double v = finish(p, b, m, n, acc[n]);
     if (out64) out64[n] = v;
     if (out16) put(p, out16, n, v);
+    acc[n] = v;                                  // kept for the row reduction below
+  }
+  if (reduce_op != REDUCE_NONE && reduced) {
+    double mx = acc[0];
+    for (int64_t n = 1; n < p.N; ++n) mx = acc[n] > mx ? acc[n] : mx;
+    double r = 0.0;
+    if (reduce_op == REDUCE_SUM) {
+      for (int64_t n = 0; n < p.N; ++n) r += acc[n];
+    } else if (reduce_op == REDUCE_MAX) {
+      r = mx;
+    } else {
+      for (int64_t n = 0; n < p.N; ++n) r += std::exp(acc[n] - mx);
+      r = mx + std::log(r);
+    }
+    *reduced = r;
   }
 }
 
@@ -355,6 +375,29 @@ int cg_ref_diag_matmul(const float* d, const void* B, double* c64, void* cout, i
         else static_cast<uint16_t*>(cout)[i * N + j] = f64_to_bf16_rne(v);
       }
     }
+  return 0;
+}
+
+// Extended family with a fused row reduction: as cg_ref_gemm_epilogue_ex, plus reduced[i] = the reduction of
+// row i's N values (reduce_op 1 sum, 2 max, 3 logsumexp).  d64 and dout may be NULL.
+int cg_ref_gemm_epilogue_reduce(const void* A, const void* B, const void* bias, const void* R, const int64_t* rows,
+                                int64_t nrows, double* d64, void* dout, double* reduced, int reduce_op, int64_t M, int64_t N,
+                                int64_t K, int64_t batch, double alpha, double beta, int act, const float* row_scale,
+                                const float* col_scale, double clamp_lo, double clamp_hi, int out_dtype) {
+  const Problem p = make_ex(A, B, bias, R, M, N, K, batch, alpha, beta, act, row_scale, col_scale, clamp_lo, clamp_hi,
+                            out_dtype);
+  if (bad(p) || out_dtype < OUT_BF16 || out_dtype > OUT_F32 || (p.clamp && !(clamp_lo <= clamp_hi)) || !reduced ||
+      reduce_op < REDUCE_SUM || reduce_op > REDUCE_LOGSUMEXP)
+    return 1;
+  if (!rows) nrows = batch * M;
+  const int64_t esize = out_dtype == OUT_F32 ? 4 : 2;
+  std::vector<double> acc(static_cast<size_t>(N));
+  for (int64_t i = 0; i < nrows; ++i) {
+    const int64_t r = rows ? rows[i] : i;
+    if (r < 0 || r >= batch * M) return 1;
+    row(p, r / M, r % M, acc, d64 ? d64 + i * N : nullptr, dout ? static_cast<char*>(dout) + i * N * esize : nullptr,
+        reduce_op, reduced + i);
+  }
   return 0;
 }
 

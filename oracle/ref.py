@@ -24,6 +24,7 @@ FLAG_B_BROADCAST = 1 << 11
 FLAG_CLAMP = 1 << 12
 FLAG_IN_F32 = 1 << 13
 OUT_BF16, OUT_F16, OUT_F32 = 0, 1, 2
+REDUCE_SUM, REDUCE_MAX, REDUCE_LOGSUMEXP = 1, 2, 3
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "cg_oracle.cpp")
@@ -73,6 +74,9 @@ def _load():
         lib.cg_ref_gemm_epilogue_ex.argtypes = [vp, vp, vp, vp, vp, i64, vp, vp, i64, i64, i64, i64, dbl, dbl, ci, vp, vp,
                                                 dbl, dbl, ci]
         lib.cg_ref_gemm_epilogue_ex.restype = ci
+        lib.cg_ref_gemm_epilogue_reduce.argtypes = [vp, vp, vp, vp, vp, i64, vp, vp, vp, ci, i64, i64, i64, i64, dbl, dbl, ci, vp, vp,
+                                                    dbl, dbl, ci]
+        lib.cg_ref_gemm_epilogue_reduce.restype = ci
         lib.cg_ref_diag_matmul.argtypes = [vp, vp, vp, vp, i64, i64, ci]
         lib.cg_ref_diag_matmul.restype = ci
         lib.cg_ref_f32_as_tf32.argtypes = [ctypes.c_float]
@@ -176,6 +180,28 @@ def gemm_epilogue_ex(A, B, bias, R, M, N, K, batch, alpha, beta, act, row_scale=
     if rc != 0:
         raise ValueError("oracle rejected the arguments")
     return d64, dout
+
+
+def gemm_epilogue_reduce(A, B, bias, R, M, N, K, batch, alpha, beta, act, reduce_op, row_scale=None, col_scale=None,
+                         clamp_lo=0.0, clamp_hi=0.0, out_dtype=OUT_BF16, rows=None):
+    """The extended epilogue with a fused reduction of every output row over its N unrounded values
+    (reduce_op: REDUCE_SUM, REDUCE_MAX, REDUCE_LOGSUMEXP).  Returns (D64, Dout, reduced [rows] float64)."""
+    r = None if rows is None else np.ascontiguousarray(rows, dtype=np.int64)
+    nrows = batch * M if r is None else r.size
+    shape = (batch, M, N) if r is None else (r.size, N)
+    d64 = np.empty(shape, dtype=np.float64)
+    dout = np.empty(shape, dtype=np.float32 if out_dtype == OUT_F32 else np.uint16)
+    red = np.empty(nrows, dtype=np.float64)
+    in_dtype = np.float32 if act & FLAG_IN_F32 else np.uint16
+    if A.dtype != in_dtype or B.dtype != in_dtype or not A.flags.c_contiguous or not B.flags.c_contiguous:
+        raise TypeError("A and B must be C-contiguous arrays of the operand type")
+    rc = _load().cg_ref_gemm_epilogue_reduce(_ptr(A), _ptr(B), _ptr(bias), _ptr(R), _ptr(r), 0 if r is None else r.size,
+                                             _ptr(d64), _ptr(dout), _ptr(red), int(reduce_op), M, N, K, batch, float(alpha),
+                                             float(beta), int(act), _ptr(row_scale), _ptr(col_scale), float(clamp_lo),
+                                             float(clamp_hi), int(out_dtype))
+    if rc != 0:
+        raise ValueError("oracle rejected the arguments")
+    return d64, dout, red
 
 
 def diag_matmul(d, B, out_dtype=OUT_BF16):

@@ -242,3 +242,64 @@ def test_tf32_small_integers_exact(oracle):
     e64, e32 = run_ex(oracle, p)
     want = np.einsum("bmk,bnk->bmn", p.A.astype(np.int64), p.B.astype(np.int64))
     assert np.array_equal(e64, want.astype(np.float64)) and np.array_equal(e32, want.astype(np.float32))
+
+
+# ---------------------------------------------------------------- fused row reduction
+
+def run_reduce(oracle, p, op, **kw):
+    return oracle.gemm_epilogue_reduce(p.A, p.B, p.bias, p.R, p.M, p.N, p.K, p.batch, p.alpha, p.beta, p.act, op,
+                                       row_scale=p.row_scale, col_scale=p.col_scale, clamp_lo=p.clamp_lo, clamp_hi=p.clamp_hi,
+                                       out_dtype=p.out_dtype, **kw)
+
+
+def test_row_reduction_closed_forms(oracle):
+    """All-ones operands: every v is K (+ bias), so sum = N*K, max = K, logsumexp = K + log N.  A = 0: v = act(bias[n])."""
+    M, N, K = 5, 24, 64
+    ones = gen.f32_to_bf16_bits(np.ones((1, M, K), dtype=np.float32)), gen.f32_to_bf16_bits(np.ones((1, K, N), dtype=np.float32))
+    for op, want in ((oracle.REDUCE_SUM, N * K), (oracle.REDUCE_MAX, K), (oracle.REDUCE_LOGSUMEXP, K + np.log(N))):
+        _, _, red = oracle.gemm_epilogue_reduce(ones[0], ones[1], None, None, M, N, K, 1, 1.0, 0.0, W.ACT_NONE, op)
+        assert np.allclose(red, want, rtol=1e-15, atol=0)
+    p = W.make(M, N, K, seed=3, act=W.ACT_SIGMOID, A=("zeros", 0.0), B=("normal", 1.0), bias=("normal", 2.0))
+    v = 1.0 / (1.0 + np.exp(-p.bias.astype(np.float64)))
+    assert np.allclose(run_reduce(oracle, p, oracle.REDUCE_SUM)[2], v.sum(), rtol=1e-14)
+    assert np.allclose(run_reduce(oracle, p, oracle.REDUCE_MAX)[2], v.max(), rtol=1e-15)
+    assert np.allclose(run_reduce(oracle, p, oracle.REDUCE_LOGSUMEXP)[2], np.log(np.exp(v).sum()), rtol=1e-14)
+
+
+def test_row_reduction_against_library_routines_and_invariants(oracle):
+    from scipy.special import logsumexp
+    M, N, K, batch = 19, 40, 48, 2
+    kw = dict(seed=17, act=W.ACT_GELU_TANH, alpha=0.5, beta=1.0, A=("normal", 1.0), B=("normal", 1.0), bias=("normal", 1.0), R=("normal", 2.0))
+    p = W.make(M, N, K, batch, **kw)
+    d64, _ = run_ex(oracle, p)                                        # the (pinned) values that are reduced
+    rows = d64.reshape(-1, N)
+    _, _, s = run_reduce(oracle, p, oracle.REDUCE_SUM)
+    _, _, mx = run_reduce(oracle, p, oracle.REDUCE_MAX)
+    d64b, dout, lse = run_reduce(oracle, p, oracle.REDUCE_LOGSUMEXP)
+    assert np.array_equal(d64b, d64)                                  # D itself is unchanged by asking for a reduction
+    assert np.allclose(s, np.sum(rows, axis=1), rtol=1e-13) and np.array_equal(mx, np.max(rows, axis=1))
+    assert np.allclose(lse, logsumexp(rows, axis=1), rtol=1e-13)
+    assert np.all(lse >= mx) and np.all(lse <= mx + np.log(N))        # max <= logsumexp <= max + log N
+    # the residual enters the sum linearly: sum with R minus sum without = beta * sum_n R
+    q = W.make(M, N, K, batch, **dict(kw, beta=0.0))
+    _, _, s0 = run_reduce(oracle, q, oracle.REDUCE_SUM)
+    assert np.allclose(s - s0, f64(p.R).reshape(-1, N).sum(axis=1), rtol=1e-10, atol=1e-10)
+    # shifting every value of a row by a constant shifts its logsumexp by the same constant (per-row bias, no activation)
+    base = W.make(M, N, K, seed=18, act=W.ACT_NONE | W.FLAG_BIAS_PER_ROW, A=("normal", 1.0), B=("normal", 1.0), bias=("zeros", 0.0))
+    shifted = W.make(M, N, K, seed=18, act=W.ACT_NONE | W.FLAG_BIAS_PER_ROW, A=("normal", 1.0), B=("normal", 1.0), bias=("normal", 3.0))
+    l0 = run_reduce(oracle, base, oracle.REDUCE_LOGSUMEXP)[2]
+    l1 = run_reduce(oracle, shifted, oracle.REDUCE_LOGSUMEXP)[2]
+    assert np.allclose(l1 - l0, shifted.bias.astype(np.float64), rtol=1e-12, atol=1e-12)
+    # the reduction sees the unrounded values, not the stored bf16 ones
+    assert not np.allclose(s, np.sum(f64(dout).reshape(-1, N), axis=1), rtol=1e-9, atol=0)
+    # selected rows
+    sel = np.array([0, 7, M, batch * M - 1])
+    assert np.array_equal(run_reduce(oracle, p, oracle.REDUCE_SUM, rows=sel)[2], s[sel])
+
+
+def test_row_reduction_large_values_do_not_overflow(oracle):
+    M, N, K = 3, 16, 8
+    p = W.make(M, N, K, seed=1, act=W.ACT_NONE, alpha=1.0, A=("zeros", 0.0), B=("zeros", 0.0), bias=("normal", 400.0))
+    lse = run_reduce(oracle, p, oracle.REDUCE_LOGSUMEXP)[2]
+    b = p.bias.astype(np.float64)
+    assert np.all(np.isfinite(lse)) and np.allclose(lse, b.max() + np.log(np.exp(b - b.max()).sum()), rtol=1e-15)
