@@ -345,16 +345,24 @@ def extended_sweep(ctx, p, dev, flush):
         "clamp": dict(act=p.act | FLAG_CLAMP, clamp_lo=-0.5, clamp_hi=2.0),
         "out_f16": dict(D=d16, out_dtype=1),
         "out_f32": dict(D=d32, out_dtype=2),
+        "row_sum": dict(row_reduce=1, row_out=rs),
+        "row_logsumexp": dict(row_reduce=3, row_out=rs),
+        "row_logsumexp_without_D": dict(D=None, row_reduce=3, row_out=rs),
     }
     out = {}
     for label, v in variants.items():
         v = dict(v)
-        D = v.pop("D", dev["D"])
+        D = v.pop("D") if "D" in v else dev["D"]
         act = v.pop("act", p.act)
         call = lambda: ctx.gemm_epilogue_ex(dev["A"], dev["B"], dev["bias"], dev["R"], D, p.M, p.N, p.K, p.batch, p.alpha, p.beta, act, **v)
         timed(call, 2, flush)
         out[label] = min(timed(call, 10, flush)) * 1e6
     ctx.check()
+    # the unfused form of the last variants: GEMM + bias + GELU, then a row-wise logsumexp over the stored tensor
+    import torch.nn.functional as F
+    unfused = lambda: torch.logsumexp(F.gelu(torch.matmul(dev["A"][0], dev["B"][0]) + dev["bias"].to(torch.bfloat16), approximate="tanh").float(), dim=1)
+    timed(unfused, 2, flush)
+    out["torch_eager_gemm_gelu_logsumexp"] = min(timed(unfused, 5, flush)) * 1e6
     return out
 
 

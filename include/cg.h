@@ -113,15 +113,27 @@ CG_API int cg_gemm_epilogue(cg_handle_t h, const void* A, const void* B, const v
  *                         shared by all batch entries
  *   out_dtype             element type of D: CG_OUT_BF16, CG_OUT_F16 or CG_OUT_F32 (R stays bf16); D must be
  *                         16-byte aligned and N % 8 == 0 as before
- * Errors as for cg_gemm_epilogue; CG_ERR_INVALID_ARG also for clamp_lo > clamp_hi or CG_FLAG_CLAMP without ex.
+ *   row_reduce, row_out   fused reduction epilogue (the prompt's "Fuse reduction epilogue", consumers sum / max /
+ *                         logsumexp): row_out[b*M + m] = sum_n v, max_n v or log(sum_n exp(v)) over the N values
+ *                         v = u + beta*R of the row, taken in fp32 before they are rounded for storage.  D may be
+ *                         NULL when only the reduction is wanted (then no output tensor is written at all).
+ *                         Two launches: the GEMM kernel leaves one partial per row, tile column and epilogue warp
+ *                         in a scratch buffer owned by the handle (grown with cudaMalloc when a call needs more
+ *                         than any before it), a second small kernel combines them in a fixed order, so the
+ *                         result is deterministic.
+ * Errors as for cg_gemm_epilogue; CG_ERR_INVALID_ARG also for clamp_lo > clamp_hi, CG_FLAG_CLAMP without ex, an
+ * unknown row_reduce code or a reduction without row_out.
  */
 enum { CG_FLAG_BIAS_PER_ROW = 1 << 10, CG_FLAG_B_BROADCAST = 1 << 11, CG_FLAG_CLAMP = 1 << 12, CG_FLAG_IN_F32 = 1 << 13 };
 enum { CG_OUT_BF16 = 0, CG_OUT_F16 = 1, CG_OUT_F32 = 2 };
+enum { CG_REDUCE_NONE = 0, CG_REDUCE_SUM = 1, CG_REDUCE_MAX = 2, CG_REDUCE_LOGSUMEXP = 3 };
 typedef struct cg_epilogue_ex {
   const float* row_scale;
   const float* col_scale;
   float clamp_lo, clamp_hi;
   int out_dtype;
+  int row_reduce;  /* CG_REDUCE_*: fused reduction of every output row, see below */
+  float* row_out;  /* device, fp32 [batch*M]: the reduced values */
 } cg_epilogue_ex_t;
 CG_API int cg_gemm_epilogue_ex(cg_handle_t h, const void* A, const void* B, const void* bias, const void* R, void* D,
                                int M, int N, int K, int batch, float alpha, float beta, int act,
@@ -195,7 +207,7 @@ typedef struct cg_plan_info {
   int dp_units;    /* leading units that are whole tiles     */
   int k_blocks;    /* 64-wide k-blocks per tile              */
   int smem_bytes;  /* dynamic shared memory per CTA          */
-  int launches;    /* kernels launched by the call (always 1)*/
+  int launches;    /* kernels launched by the call: 1, or 2 with a fused row reduction */
   int cluster_split; /* K parts per tile held by one cluster (1 = off) */
   int latency_kernel; /* 1: the short single-tile-per-CTA kernel for small problems ran (every tile on its own SM,
                          K <= 512, at most 2^19 outputs, base epilogue, no plan override) */

@@ -22,6 +22,7 @@ CG_FLAG_B_BROADCAST = 1 << 11
 CG_FLAG_CLAMP = 1 << 12
 CG_FLAG_IN_F32 = 1 << 13
 CG_OUT_BF16, CG_OUT_F16, CG_OUT_F32 = 0, 1, 2
+CG_REDUCE_NONE, CG_REDUCE_SUM, CG_REDUCE_MAX, CG_REDUCE_LOGSUMEXP = 0, 1, 2, 3
 
 STATUS_NAMES = {0: "CG_OK", 1: "CG_ERR_INVALID_ARG", 2: "CG_ERR_UNSUPPORTED", 3: "CG_ERR_ARCH", 4: "CG_ERR_CUDA",
                 5: "CG_ERR_WORKSPACE", 6: "CG_ERR_TIMEOUT"}
@@ -36,7 +37,7 @@ class cg_tuning_t(ctypes.Structure):
 
 class cg_epilogue_ex_t(ctypes.Structure):
     _fields_ = [("row_scale", ctypes.c_void_p), ("col_scale", ctypes.c_void_p), ("clamp_lo", ctypes.c_float),
-                ("clamp_hi", ctypes.c_float), ("out_dtype", ctypes.c_int)]
+                ("clamp_hi", ctypes.c_float), ("out_dtype", ctypes.c_int), ("row_reduce", ctypes.c_int), ("row_out", ctypes.c_void_p)]
 
 
 class cg_plan_info_t(ctypes.Structure):
@@ -146,9 +147,11 @@ def cg_gemm_epilogue(h, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, stre
 
 
 def cg_gemm_epilogue_ex(h, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, row_scale=None, col_scale=None, clamp_lo=0.0,
-                        clamp_hi=0.0, out_dtype=CG_OUT_BF16, stream=None) -> int:
-    """The wider consumer family (scale vectors, per-row bias, clamp, shared B, bf16 / fp16 / fp32 output)."""
-    ex = cg_epilogue_ex_t(_dev_ptr(row_scale), _dev_ptr(col_scale), float(clamp_lo), float(clamp_hi), int(out_dtype))
+                        clamp_hi=0.0, out_dtype=CG_OUT_BF16, row_reduce=CG_REDUCE_NONE, row_out=None, stream=None) -> int:
+    """The wider consumer family (scale vectors, per-row bias, clamp, shared B, bf16 / fp16 / fp32 output, fp32 / TF32
+    operands, fused row reduction into ``row_out``; D may be None when only the reduction is wanted)."""
+    ex = cg_epilogue_ex_t(_dev_ptr(row_scale), _dev_ptr(col_scale), float(clamp_lo), float(clamp_hi), int(out_dtype),
+                          int(row_reduce), _dev_ptr(row_out))
     return load().cg_gemm_epilogue_ex(h, _dev_ptr(A), _dev_ptr(B), _dev_ptr(bias), _dev_ptr(R), _dev_ptr(D), int(M), int(N),
                                       int(K), int(batch), float(alpha), float(beta), int(act), ctypes.byref(ex),
                                       _stream_ptr(stream))

@@ -87,6 +87,7 @@ struct cg_context {
   MapCacheEntry map_cache[MAP_CACHE_SIZE];
   int map_cache_next = 0;
   StagingBuf sA, sB, sBias, sR, sD;
+  StagingBuf row_ws;                     // partial results of fused row reductions
   std::mutex mu;
 };
 
@@ -425,11 +426,15 @@ int launch_small(cg_context* h, const void* A, const void* B, const void* bias, 
   return CG_OK;
 }
 
+int grow(cg_context* h, StagingBuf* s, size_t bytes);
+
 int launch(cg_context* h, const void* A, const void* B, const void* bias, const void* R, void* D, int M, int N, int K,
            int batch, float alpha, float beta, int act, cudaStream_t stream, const cg_epilogue_ex_t* ex = nullptr) {
   const bool b_kmajor = (act & CG_FLAG_B_COLMAJOR) != 0;
   const bool ext_in_use = (act & (CG_FLAG_BIAS_PER_ROW | CG_FLAG_B_BROADCAST | CG_FLAG_CLAMP | CG_FLAG_IN_F32)) != 0 ||
-                          (ex && (ex->row_scale || ex->col_scale || ex->out_dtype != CG_OUT_BF16));
+                          (ex && (ex->row_scale || ex->col_scale || ex->out_dtype != CG_OUT_BF16 || ex->row_reduce));
+  const int row_reduce = ex ? ex->row_reduce : 0;
+  const bool store_d = D != nullptr;
   if (!ext_in_use) {
     const int rs = launch_small(h, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, stream);
     if (rs >= 0) return rs;
@@ -441,7 +446,7 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   const bool tf32 = (act & CG_FLAG_IN_F32) != 0;
   const int bk_elems = tf32 ? BK / 2 : BK;
   const int in_dtype = tf32 ? CG_OUT_F32 : CG_OUT_BF16;           // (element type code of A and B)
-  int rc = make_plan(h, M, N, K, batch, b_kmajor, beta != 0.0f, &pl, out_dtype == CG_OUT_F32, bk_elems);
+  int rc = make_plan(h, M, N, K, batch, b_kmajor, beta != 0.0f, &pl, out_dtype == CG_OUT_F32 || !store_d, bk_elems);
   if (rc != CG_OK) return rc;
   KernelEntry e;
   lookup(pl.bn, pl.cg, b_kmajor, &e);
@@ -452,8 +457,13 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   if (b_kmajor) rc = make_map(h, &tmB, B, K, N, b_entries, bk_elems, e.sub_cols, in_dtype);
   else rc = make_map(h, &tmB, B, N, K, b_entries, 64, BK);
   if (rc != CG_OK) return rc;
-  if ((rc = make_map(h, &tmD, D, N, M, batch, out_dtype == CG_OUT_F32 ? 32 : EPI_COLS, 32, out_dtype)) != CG_OK) return rc;
-  if ((rc = make_map(h, &tmR, beta != 0.0f ? R : D, N, M, batch, EPI_COLS, 32)) != CG_OK) return rc;   // unused without a residual
+  if (store_d) rc = make_map(h, &tmD, D, N, M, batch, out_dtype == CG_OUT_F32 ? 32 : EPI_COLS, 32, out_dtype);
+  else rc = make_map(h, &tmD, A, tf32 ? 2 * K : K, M, batch, EPI_COLS, 32);          // never used: any valid 16-bit view
+  if (rc != CG_OK) return rc;
+  // (unused without a residual)
+  if ((rc = make_map(h, &tmR, beta != 0.0f ? R : (store_d ? D : A), beta != 0.0f || store_d ? N : (tf32 ? 2 * K : K), M, batch,
+                     EPI_COLS, 32)) != CG_OK)
+    return rc;
 
   KernelParams p;
   memset(&p, 0, sizeof p);
@@ -492,7 +502,16 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
     p.row_scale = ex->row_scale;
     p.col_scale = ex->col_scale;
   }
-  p.ext = (p.bias_per_row || p.clamp || out_dtype != CG_OUT_BF16 || p.row_scale || p.col_scale) ? 1 : 0;   // (epilogue only)
+  p.row_reduce = row_reduce;
+  p.store_d = store_d ? 1 : 0;
+  if (row_reduce) {
+    const int col_groups = e.threads > 192 ? 2 : 1;            // epilogue warps per TMEM lane quarter
+    p.row_slots = pl.tiles_n * (pl.cluster_split > 1 ? pl.cluster_split : 1) * col_groups;
+    const size_t need = static_cast<size_t>(batch) * M * p.row_slots * (row_reduce == CG_REDUCE_LOGSUMEXP ? 8 : 4);
+    if ((rc = grow(h, &h->row_ws, need)) != CG_OK) return rc;
+    p.row_ws = static_cast<float*>(h->row_ws.ptr);
+  }
+  p.ext = (p.bias_per_row || p.clamp || out_dtype != CG_OUT_BF16 || p.row_scale || p.col_scale || row_reduce) ? 1 : 0;   // (epilogue only)
   p.R = (beta != 0.0f) ? static_cast<const __nv_bfloat16*>(R) : nullptr;
   p.partials = h->partials;
   p.tickets = h->tickets;
@@ -515,12 +534,17 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   cfg.numAttrs = (attr[0].val.clusterDim.x > 1 || getenv("CG_ALWAYS_CLUSTER")) ? 1 : 0;      // a plain launch when there is no cluster
   void* args[5] = {&tmA, &tmB, &tmD, &tmR, &p};
   CG_CUDA(h, cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(e.fn), args));
+  if (row_reduce) {
+    const long long rows = static_cast<long long>(batch) * M;
+    row_finalize_kernel<<<static_cast<unsigned>((rows + 255) / 256), 256, 0, stream>>>(p.row_ws, ex->row_out, rows, p.row_slots, row_reduce);
+    CG_CUDA(h, cudaGetLastError());
+  }
 
   cg_plan_info_t& lp = h->last_plan;
   lp.tile_m = BM * pl.cg; lp.tile_n = pl.bn; lp.cta_group = pl.cg; lp.stages = pl.stages; lp.group_m = pl.group_m;
   lp.grid = pl.grid; lp.num_tiles = pl.num_tiles; lp.num_units = pl.num_units; lp.dp_units = pl.dp_units;
   lp.k_blocks = pl.k_blocks;
-  lp.smem_bytes = pl.smem; lp.launches = 1; lp.cluster_split = pl.cluster_split; lp.latency_kernel = 0;
+  lp.smem_bytes = pl.smem; lp.launches = row_reduce ? 2 : 1; lp.cluster_split = pl.cluster_split; lp.latency_kernel = 0;
   h->last_status = CG_OK;
   h->last_msg[0] = 0;
   if (h->log_plans)
@@ -609,12 +633,18 @@ int cg_gemm_epilogue_ex(cg_handle_t h, const void* A, const void* B, const void*
                         int N, int K, int batch, float alpha, float beta, int act, const cg_epilogue_ex_t* ex, void* stream) {
   if (!h) return CG_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lock(h->mu);
-  int rc = validate(h, A, B, bias, R, D, M, N, K, batch, beta, act,
+  const bool reducing = ex && ex->row_reduce != CG_REDUCE_NONE;
+  if (ex && (ex->row_reduce < CG_REDUCE_NONE || ex->row_reduce > CG_REDUCE_LOGSUMEXP || (reducing && !ex->row_out) ||
+             (reducing && (reinterpret_cast<uintptr_t>(ex->row_out) & 3))))
+    return fail(h, CG_ERR_INVALID_ARG, "row_reduce must be a CG_REDUCE_* code with a 4-byte aligned row_out");
+  // with a row reduction D may be NULL (only the reduction is wanted)
+  int rc = validate(h, A, B, bias, R, (!D && reducing) ? const_cast<void*>(A) : D, M, N, K, batch, beta, act,
                     CG_FLAG_BIAS_PER_ROW | CG_FLAG_B_BROADCAST | CG_FLAG_CLAMP | CG_FLAG_IN_F32);
   if (rc != CG_OK) return rc;
   if ((act & CG_FLAG_IN_F32) && !(act & CG_FLAG_B_COLMAJOR))
     return fail(h, CG_ERR_UNSUPPORTED, "fp32 operands need B stored [batch,N,K] (CG_FLAG_B_COLMAJOR)");
-  if ((rc = check_alignment(h, A, B, (act & CG_FLAG_BIAS_PER_ROW) ? nullptr : bias, R, D, beta, act)) != CG_OK) return rc;
+  if ((rc = check_alignment(h, A, B, (act & CG_FLAG_BIAS_PER_ROW) ? nullptr : bias, R, D ? D : const_cast<void*>(A), beta, act)) != CG_OK)
+    return rc;
   if (ex) {
     if (ex->out_dtype < CG_OUT_BF16 || ex->out_dtype > CG_OUT_F32) return fail(h, CG_ERR_INVALID_ARG, "unknown output dtype %d", ex->out_dtype);
     if ((reinterpret_cast<uintptr_t>(ex->row_scale) | reinterpret_cast<uintptr_t>(ex->col_scale)) & 3)
@@ -742,7 +772,7 @@ int cg_destroy(cg_handle_t h) {
   cudaSetDevice(h->device);
   cudaFree(h->workspace);
   cudaFree(h->status);
-  StagingBuf* bufs[5] = {&h->sA, &h->sB, &h->sBias, &h->sR, &h->sD};
+  StagingBuf* bufs[6] = {&h->sA, &h->sB, &h->sBias, &h->sR, &h->sD, &h->row_ws};
   for (StagingBuf* s : bufs)
     if (s->ptr) cudaFree(s->ptr);
   delete h;

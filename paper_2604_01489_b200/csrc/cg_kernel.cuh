@@ -66,6 +66,7 @@ constexpr int CTRL_BYTES = 256;
 enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU_TANH = 2, ACT_SILU = 3,
        ACT_GELU_ERF = 4, ACT_SIGMOID = 5, ACT_TANH = 6, ACT_LEAKY_RELU = 7 };
 enum { OUT_BF16 = 0, OUT_F16 = 1, OUT_F32 = 2 };
+enum { REDUCE_NONE = 0, REDUCE_SUM = 1, REDUCE_MAX = 2, REDUCE_LOGSUMEXP = 3 };
 enum { STATUS_OK = 0, STATUS_SMEM = 4, STATUS_TIMEOUT = 6 };
 
 struct KernelParams {
@@ -95,6 +96,10 @@ struct KernelParams {
   int b_broadcast;        // one B shared by all batch entries
   int clamp;              // clamp the activation's result to [clamp_lo, clamp_hi]
   int out_dtype;          // OUT_BF16 / OUT_F16 / OUT_F32
+  int row_reduce;         // REDUCE_*: every row's N final values are also reduced (partials to row_ws, see row_finalize_kernel)
+  int store_d;            // 0: D is not wanted, only the row reduction
+  int row_slots;          // partial results per row: tiles_n x K parts of a cluster x column groups
+  float* row_ws;          // [batch*M][row_slots] (two floats per slot for logsumexp: running maximum, scaled sum)
   int tf32;               // A and B are fp32 and multiplied as TF32: a k-block is 32 elements (still 128 bytes),
                           // one MMA covers 8 of them; B is K-major
   float clamp_lo, clamp_hi;
@@ -764,6 +769,8 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           cs_reg[2 * j + 1] = (p.col_scale != nullptr && col + 32 < p.N) ? __ldg(p.col_scale + col + 32) : 1.0f;
         }
       }
+      // fused row reduction: this thread's row, this warp's columns of the tile
+      float red_m = -INFINITY, red_s = 0.0f;
       if (!dry && !wait_bar(ptx::smem_u32(&ctrl->acc_full[acc]), acc_phase, ctrl, p)) { ok = false; break; }
       if (!dry && ew == 0 && lane == 0) trace_event(p, TR_ACC_SEEN);
       ptx::tc_fence_after();
@@ -934,6 +941,29 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
               default: finalize_chunk_ext<ACT_NONE>(accv, bias_s, row_mul, row_bias, cs_reg[2 * c_ord], cs_reg[2 * c_ord + 1], p, has_r, rq); break;
             }
 #undef CG_EXT_CASE
+            if (p.row_reduce) {
+              const int nvalid = p.N - n0 < EPI_COLS ? p.N - n0 : EPI_COLS;     // columns of this chunk that exist
+              if (p.row_reduce == REDUCE_SUM) {
+#pragma unroll
+                for (int j = 0; j < EPI_COLS; ++j) red_s += (j < nvalid) ? accv[j] : 0.0f;
+              } else {
+                float cm = -INFINITY;
+#pragma unroll
+                for (int j = 0; j < EPI_COLS; ++j) cm = (j < nvalid) ? fmaxf(cm, accv[j]) : cm;
+                if (p.row_reduce == REDUCE_LOGSUMEXP) {
+                  // running (maximum, sum of exp(v - maximum)): rescale the old sum, add this chunk's terms
+                  const float nm = fmaxf(red_m, cm);
+                  float add = 0.0f;
+#pragma unroll
+                  for (int j = 0; j < EPI_COLS; ++j) add += (j < nvalid) ? __expf(accv[j] - nm) : 0.0f;
+                  red_s = red_s * __expf(red_m - nm) + add;       // (red_m = -inf at first: the factor is 0)
+                  red_m = nm;
+                } else {
+                  red_m = fmaxf(red_m, cm);
+                }
+              }
+              if (!p.store_d) continue;
+            }
             if (p.out_dtype == OUT_F32) {
               // fp32 rows are 256 bytes: the chunk leaves as two 32-column boxes through the same buffer
 #pragma unroll
@@ -1000,6 +1030,18 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           store_buf = (store_buf + 1 == C::EPI_BUFS) ? 0 : store_buf + 1;
           if (r_shared && !dry) request_next_residual(c, c_step, c_hi, n0, m_base + q * 32, b, have_next, s_next, c_lo);
         }
+        if (p.row_reduce && !dry && ok) {      // this row's partial over this warp's columns (identity if it had none)
+          const int m = m_base + row_in_tile;
+          if (m < p.M) {
+            const size_t slot = (static_cast<size_t>(b) * p.M + m) * p.row_slots +
+                                (static_cast<size_t>(nt) * csk + my_part) * C::EPI_COL_GROUPS + col_group;
+            if (p.row_reduce == REDUCE_LOGSUMEXP) {
+              reinterpret_cast<float2*>(p.row_ws)[slot] = make_float2(red_m, red_s);
+            } else {
+              p.row_ws[slot] = p.row_reduce == REDUCE_SUM ? red_s : red_m;
+            }
+          }
+        }
         if (whole_tile && c_lo >= c_hi && !dry) {    // none of this warp's columns exist (ragged N): still hand the buffer back
           ptx::tc_fence_before();
           __syncwarp();
@@ -1041,6 +1083,26 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     ptx::tc_fence_after();
     ptx::tmem_dealloc<CG>(tmem_base, C::TMEM_COLS);
     if (lane == 0) trace_event(p, TR_END);
+  }
+}
+
+// Second pass of the fused row reduction: one thread per row combines its row's partials in slot order.
+__global__ void row_finalize_kernel(const float* __restrict__ ws, float* __restrict__ out, long long rows, int slots, int op) {
+  const long long row = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (row >= rows) return;
+  if (op == REDUCE_LOGSUMEXP) {
+    const float2* w = reinterpret_cast<const float2*>(ws) + row * slots;
+    float mx = -INFINITY;
+    for (int s = 0; s < slots; ++s) mx = fmaxf(mx, w[s].x);
+    float sum = 0.0f;
+    for (int s = 0; s < slots; ++s)
+      if (w[s].x > -INFINITY) sum += w[s].y * expf(w[s].x - mx);
+    out[row] = mx + logf(sum);
+  } else {
+    const float* w = ws + row * slots;
+    float acc = op == REDUCE_SUM ? 0.0f : -INFINITY;
+    for (int s = 0; s < slots; ++s) acc = op == REDUCE_SUM ? acc + w[s] : fmaxf(acc, w[s]);
+    out[row] = acc;
   }
 }
 

@@ -213,3 +213,89 @@ def test_tf32_needs_k_major_b(ctx):
     assert rc == cg.CG_ERR_UNSUPPORTED
     rc = cg.cg_gemm_epilogue(ctx.handle, a, a, None, None, d, 64, 64, 64, 1, 1.0, 0.0, cg.CG_FLAG_IN_F32 | cg.CG_FLAG_B_COLMAJOR)
     assert rc == cg.CG_ERR_INVALID_ARG                                   # the base entry point has no fp32 operands
+
+
+# ------------------------------------------------------------------ fused row reduction
+
+REDUCE_PLANS = [dict(tile_n=64, cta_group=1), dict(tile_n=128, cta_group=1), dict(tile_n=256, cta_group=1),
+                dict(tile_n=128, cta_group=2), dict(tile_n=256, cta_group=2), dict(tile_n=512, cta_group=2), dict(),
+                dict(tile_n=128, cta_group=1, num_units=29), dict(tile_n=256, cta_group=2, num_units=11),
+                dict(tile_n=128, cta_group=1, cluster_split=2), dict(tile_n=256, cta_group=1, cluster_split=4)]
+
+
+def run_reduce_gpu(ctx, p, op, store_d=True):
+    import torch
+    dev = PU.to_device_ex(p)
+    dev["D"].fill_(float("nan"))
+    out = torch.full((p.batch * p.M,), float("nan"), dtype=torch.float32, device="cuda")
+    ctx.gemm_epilogue_ex(dev["A"], dev["B"], dev["bias"], dev["R"], dev["D"] if store_d else None, p.M, p.N, p.K, p.batch, p.alpha,
+                         p.beta, p.act, row_scale=dev["row_scale"], col_scale=dev["col_scale"], clamp_lo=p.clamp_lo,
+                         clamp_hi=p.clamp_hi, out_dtype=p.out_dtype, row_reduce=op, row_out=out)
+    ctx.check()
+    return dev["D"], out.cpu().numpy().astype(np.float64)
+
+
+@pytest.mark.parametrize("plan", REDUCE_PLANS, ids=lambda d: "auto" if not d else "-".join(f"{k}{v}" for k, v in d.items()))
+def test_row_reduction_integer_operands_exact(ctx, oracle, plan):
+    """Integer values: every v is an exact fp32 integer, so row sums (< 2^24) and maxima are exact whatever the
+    order the partials are combined in; logsumexp within 1e-5 relative."""
+    import torch
+    M, N, K, batch = (300, 328, 1024, 2)
+    p = W.make(M, N, K, batch, seed=61, act=W.ACT_RELU | W.FLAG_B_COLMAJOR, alpha=1.0, beta=-1.0, A=SI, B=SI, bias=SI, R=SI,
+               clamp=(0.0, 12.0))
+    ctx.set_tuning(reset=True)
+    if plan:
+        ctx.set_tuning(**plan)
+    r64, rout, want_sum = oracle.gemm_epilogue_reduce(p.A, p.B, p.bias, p.R, M, N, K, batch, p.alpha, p.beta, p.act, oracle.REDUCE_SUM,
+                                                      clamp_lo=p.clamp_lo, clamp_hi=p.clamp_hi)
+    D, got = run_reduce_gpu(ctx, p, oracle.REDUCE_SUM)
+    assert ctx.last_plan()["launches"] == 2
+    assert np.array_equal(got, want_sum)
+    assert np.array_equal(D.view(torch.int16).cpu().numpy().view(np.uint16), rout)          # D is still written, unchanged
+    want_max = oracle.gemm_epilogue_reduce(p.A, p.B, p.bias, p.R, M, N, K, batch, p.alpha, p.beta, p.act, oracle.REDUCE_MAX,
+                                           clamp_lo=p.clamp_lo, clamp_hi=p.clamp_hi)[2]
+    D, got = run_reduce_gpu(ctx, p, oracle.REDUCE_MAX, store_d=False)
+    assert np.array_equal(got, want_max)
+    assert bool(torch.isnan(D).all()), "D was written although it was not passed"
+    want_lse = oracle.gemm_epilogue_reduce(p.A, p.B, p.bias, p.R, M, N, K, batch, p.alpha, p.beta, p.act, oracle.REDUCE_LOGSUMEXP,
+                                           clamp_lo=p.clamp_lo, clamp_hi=p.clamp_hi)[2]
+    _, got = run_reduce_gpu(ctx, p, oracle.REDUCE_LOGSUMEXP)
+    assert np.allclose(got, want_lse, rtol=1e-5, atol=1e-5)
+
+
+@pytest.mark.parametrize("op", [1, 2, 3], ids=["sum", "max", "logsumexp"])
+@pytest.mark.parametrize("act", [W.ACT_NONE, W.ACT_GELU_TANH, W.ACT_SILU])
+def test_row_reduction_random_inputs(ctx, oracle, op, act):
+    """Tolerances: max and logsumexp like an fp32 output, |r - ref| <= 2e-4 (|ref| + 1); a sum of N values carries
+    N such errors at most: |r - ref| <= 2e-4 (sum_n |v_ref| + 1)."""
+    M, N, K, batch = 333, 520, 456, 2
+    p = W.make(M, N, K, batch, seed=act + 70, act=act | W.FLAG_BIAS_BF16, alpha=0.7, beta=0.5, A=("normal", 1.0), B=("normal", 0.08),
+               bias=("normal", 1.0), R=("normal", 1.0), col_scale=("uniform", 2.0), out_dtype=W.OUT_F16)
+    d64, _, want = oracle.gemm_epilogue_reduce(p.A, p.B, p.bias, p.R, M, N, K, batch, p.alpha, p.beta, p.act, op,
+                                               col_scale=p.col_scale, out_dtype=p.out_dtype)
+    scale = np.abs(d64).reshape(-1, N).sum(axis=1) if op == 1 else np.abs(want)
+    for tuning in (dict(), dict(tile_n=256, cta_group=2), dict(tile_n=128, cta_group=1, num_units=37)):
+        ctx.set_tuning(reset=True)
+        if tuning:
+            ctx.set_tuning(**tuning)
+        _, got = run_reduce_gpu(ctx, p, op)
+        assert np.all(np.abs(got - want) <= 2e-4 * (scale + 1.0)), float(np.max(np.abs(got - want) / (scale + 1.0)))
+    _, again = run_reduce_gpu(ctx, p, op)
+    assert np.array_equal(got, again)                                                     # deterministic
+
+
+def test_row_reduction_tf32_ragged_and_errors(ctx, oracle):
+    import torch
+    import paper_2604_01489_b200 as cg
+    p = W.make(77, 1000, 136, batch=2, seed=80, act=W.ACT_NONE | TF32, A=SI, B=SI, bias=SI, out_dtype=W.OUT_F32)
+    want = oracle.gemm_epilogue_reduce(p.A, p.B, p.bias, p.R, p.M, p.N, p.K, p.batch, p.alpha, p.beta, p.act, oracle.REDUCE_SUM,
+                                       out_dtype=p.out_dtype)[2]
+    ctx.set_tuning(reset=True)
+    _, got = run_reduce_gpu(ctx, p, oracle.REDUCE_SUM)
+    assert np.array_equal(got, want)
+    a = torch.zeros(64, 64, device="cuda", dtype=torch.bfloat16)
+    out = torch.zeros(64, device="cuda")
+    h = ctx.handle
+    assert cg.cg_gemm_epilogue_ex(h, a, a, None, None, a, 64, 64, 64, 1, 1.0, 0.0, 0, row_reduce=4, row_out=out) == cg.CG_ERR_INVALID_ARG
+    assert cg.cg_gemm_epilogue_ex(h, a, a, None, None, a, 64, 64, 64, 1, 1.0, 0.0, 0, row_reduce=1, row_out=None) == cg.CG_ERR_INVALID_ARG
+    assert cg.cg_gemm_epilogue_ex(h, a, a, None, None, None, 64, 64, 64, 1, 1.0, 0.0, 0) == cg.CG_ERR_INVALID_ARG   # no D, no reduction
