@@ -38,11 +38,11 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
 # summarised under profiles/ (one capture per workload, heuristic plan).
 NCU_DRAM_TRAFFIC = {
-    "cfg1_256_relu": 0.34e6,
-    "cfg2_4096_gelu": 111.5e6,
-    "cfg3_skinny_silu": 143.6e6,
-    "cfg4_batched_residual": 251.3e6,
-    "cfg5_8192_silu": 983.3e6,
+    "cfg1_256_relu": 0.29e6,
+    "cfg2_4096_gelu": 130.7e6,
+    "cfg3_skinny_silu": 141.4e6,
+    "cfg4_batched_residual": 254.6e6,
+    "cfg5_8192_silu": 981.6e6,
 }
 
 BOUND = {"cfg1_256_relu": "latency", "cfg2_4096_gelu": "tensor", "cfg3_skinny_silu": "hbm",
