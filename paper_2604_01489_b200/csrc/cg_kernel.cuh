@@ -2,22 +2,28 @@
 //
 //   D[b,m,n] = act( alpha * sum_k A[b,m,k] * B[b,k,n] + bias[n] ) + beta * R[b,m,n]
 //
-// Roles inside one CTA of 192 threads:
+// (and, through the extended entry point, row / column scale vectors, a per-row bias, a clamp, one B
+// shared by the batch, fp16 / fp32 output, fp32 operands multiplied as TF32, and a fused reduction of
+// every output row).
+//
+// Roles inside one CTA of 64 + 32 * EPI_WARPS threads (EPI_WARPS = 4 for 64-wide tiles, else 8):
 //   warp 0 (one lane)  producer: TMA loads of A and B k-blocks into an N-stage shared-memory
 //                      ring, completion counted in bytes on `full[stage]` mbarriers;
-//   warp 1 (one lane)  MMA issuer: tcgen05.mma (bf16 x bf16 -> fp32) from the ring into one of
-//                      two accumulator buffers in tensor memory; tcgen05.commit frees ring
-//                      stages (`empty[stage]`) and publishes accumulators (`acc_full[buf]`);
-//                      the whole warp allocates / frees tensor memory;
-//   warps 2-5          epilogue: TMEM -> registers, alpha*acc + bias, activation, + beta*R,
-//                      round to bf16, swizzled shared-memory staging, TMA store.  D is written
-//                      once and never read.  Each warp owns the 32 accumulator rows (TMEM
-//                      lanes) of its quarter and never synchronises with the other warps.
+//   warp 1 (one lane)  MMA issuer: tcgen05.mma (bf16 x bf16 or TF32 x TF32 -> fp32) from the ring into
+//                      an accumulator buffer in tensor memory; tcgen05.commit frees ring stages
+//                      (`empty[stage]`) and publishes accumulators (`acc_full[buf]`); the whole
+//                      warp allocates / frees tensor memory;
+//   warps 2 and up     epilogue: TMEM -> registers, alpha*acc + bias, activation, + beta*R,
+//                      rounding, swizzled shared-memory staging, TMA store.  D is written once and
+//                      never read.  A warp owns the 32 accumulator rows (TMEM lanes) of its quarter
+//                      and, with eight warps, one half of the tile's columns; it never synchronises
+//                      with the other warps.
 //
 // Work decomposition: the iteration space (tile, k-block) is linearised tile-major and cut
 // into `num_units` contiguous ranges: the first `dp_units` are whole tiles (the full waves of a
 // data-parallel schedule), the rest divide the remaining iterations evenly (the partial last
-// wave, spread over all workers); worker w takes units w, w + W, ...  A unit that covers whole
+// wave, spread over all workers); worker w takes units w, w + W, ... -- from the highest index
+// down when there are both kinds, so that the split units run first.  A unit that covers whole
 // tiles is plain data-parallel work; a unit boundary inside a tile makes that tile
 // split-K / stream-K: every contributor writes its fp32 partial to the workspace,
 // draws a ticket, and the last one to arrive sums all partials in unit order (deterministic)
@@ -35,8 +41,7 @@
 // epilogue work is spread over all S CTAs.
 //
 // BN == 512 (CTA pairs only) is the wide form for large compute-bound problems: two N = 256 MMAs
-// per 16-wide k-step share one A operand, which cuts the bytes fetched from L2 per flop by a
-// quarter (the L2-to-SM path, not the tensor pipe, is what stalls the 256 x 256 form).  Its
+// per k-step share one A operand, which cuts the bytes fetched per flop by a quarter.  Its
 // accumulator fills all 512 TMEM columns, so it is single-buffered and eight epilogue warps
 // (two per TMEM lane quarter, half the columns each) drain it.
 //
