@@ -401,6 +401,44 @@ int cg_ref_gemm_epilogue_reduce(const void* A, const void* B, const void* bias, 
   return 0;
 }
 
+// Convolution with the fused epilogue, straight from its definition (stride 1, zero padding, NHWC; the paper's
+// canonical fused workload "convolution followed by bias addition and an activation"):
+//   y[n,oh,ow,oc] = act( alpha * sum_{kh,kw,ic} x[n, oh+kh-pad_h, ow+kw-pad_w, ic] * w[oc,kh,kw,ic] + bias[oc] ) + beta * R[n,oh,ow,oc]
+// x, w, R: bf16 bits; bias fp32 or bf16 (flag); y64 fp64 and y16 bf16 bits, each may be NULL.  Taps are summed in the
+// order kh, kw, ic.
+int cg_ref_conv2d(const uint16_t* x, const uint16_t* w, const void* bias, const uint16_t* R, double* y64, uint16_t* y16,
+                  int64_t n_img, int64_t H, int64_t W, int64_t IC, int64_t OC, int64_t KH, int64_t KW, int64_t pad_h,
+                  int64_t pad_w, double alpha, double beta, int act) {
+  const int64_t OH = H + 2 * pad_h - KH + 1, OW = W + 2 * pad_w - KW + 1;
+  const int kind = act & 0xFF;
+  if (!x || !w || n_img < 1 || H < 1 || W < 1 || IC < 1 || OC < 1 || KH < 1 || KW < 1 || pad_h < 0 || pad_w < 0 || OH < 1 ||
+      OW < 1 || kind > ACT_LAST || (beta != 0.0 && !R))
+    return 1;
+  const bool bias_bf16 = (act & FLAG_BIAS_BF16) != 0;
+  for (int64_t n = 0; n < n_img; ++n)
+    for (int64_t oh = 0; oh < OH; ++oh)
+      for (int64_t ow = 0; ow < OW; ++ow)
+        for (int64_t oc = 0; oc < OC; ++oc) {
+          double s = 0.0;
+          for (int64_t kh = 0; kh < KH; ++kh)
+            for (int64_t kw = 0; kw < KW; ++kw) {
+              const int64_t ih = oh + kh - pad_h, iw = ow + kw - pad_w;
+              if (ih < 0 || ih >= H || iw < 0 || iw >= W) continue;       // zero padding
+              const uint16_t* xp = x + ((n * H + ih) * W + iw) * IC;
+              const uint16_t* wp = w + ((oc * KH + kh) * KW + kw) * IC;
+              for (int64_t ic = 0; ic < IC; ++ic) s += bf16_to_f64(xp[ic]) * bf16_to_f64(wp[ic]);
+            }
+          double bv = 0.0;
+          if (bias) bv = bias_bf16 ? bf16_to_f64(static_cast<const uint16_t*>(bias)[oc]) : static_cast<double>(static_cast<const float*>(bias)[oc]);
+          double v = activation(kind, alpha * s + bv);
+          const int64_t o = ((n * OH + oh) * OW + ow) * OC + oc;
+          if (beta != 0.0) v += beta * bf16_to_f64(R[o]);
+          if (y64) y64[o] = v;
+          if (y16) y16[o] = f64_to_bf16_rne(v);
+        }
+  return 0;
+}
+
 // Helpers exposed so the pins can exercise them directly.
 uint16_t cg_ref_f64_to_f16(double v) { return f64_to_f16_rne(v); }
 double cg_ref_f32_as_tf32(float f) { return f32_as_tf32(f); }
