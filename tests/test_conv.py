@@ -1,0 +1,154 @@
+"""Convolution as an implicit GEMM (stride 1, NHWC) with the fused epilogue: pins for the oracle (CPU) and GPU
+parity through the C ABI."""
+import numpy as np
+import pytest
+
+from cg_inputs import gen, workloads as W
+
+SI = "smallint"
+
+
+def f64(b):
+    return gen.bf16_bits_to_f32(b).astype(np.float64)
+
+
+def problem(n, H, Wd, IC, OC, KH, KW, seed, dist=("normal", 1.0), wdist=("normal", 0.2), bias=True, residual=False, ph=0, pw=0):
+    x = gen.tensor(seed, gen.TENSOR_A, (n, H, Wd, IC), dist[0], dist[1])
+    w = gen.tensor(seed, gen.TENSOR_B, (OC, KH, KW, IC), wdist[0], wdist[1])
+    b = gen.tensor(seed, gen.TENSOR_BIAS, (OC,), dist[0], dist[1], dtype="f32") if bias else None
+    OH, OW = H + 2 * ph - KH + 1, Wd + 2 * pw - KW + 1
+    r = gen.tensor(seed, gen.TENSOR_R, (n, OH, OW, OC), dist[0], dist[1]) if residual else None
+    return x, w, b, r
+
+
+# ---------------------------------------------------------------- oracle pins (no GPU)
+
+@pytest.mark.parametrize("geom", [(2, 9, 11, 8, 16, 3, 3, 1, 1), (1, 7, 6, 16, 8, 1, 1, 0, 0), (1, 8, 8, 8, 8, 5, 3, 2, 0),
+                                  (2, 6, 10, 24, 8, 2, 4, 1, 3)], ids=str)
+def test_oracle_conv_against_torch_fp64(oracle, geom):
+    import torch
+    n, H, Wd, IC, OC, KH, KW, ph, pw = geom
+    x, w, b, r = problem(n, H, Wd, IC, OC, KH, KW, seed=sum(geom), residual=True, ph=ph, pw=pw)
+    y64, y16 = oracle.conv2d(x, w, b, r, ph, pw, alpha=0.75, beta=-0.5, act=W.ACT_NONE)
+    xt = torch.from_numpy(f64(x)).permute(0, 3, 1, 2)                     # NCHW
+    wt = torch.from_numpy(f64(w)).permute(0, 3, 1, 2)                     # [OC, IC, KH, KW]
+    ref = 0.75 * torch.nn.functional.conv2d(xt, wt, None, stride=1, padding=(ph, pw)) + torch.from_numpy(b.astype(np.float64))[None, :, None, None]
+    ref = ref.permute(0, 2, 3, 1).numpy() - 0.5 * f64(r)
+    assert y64.shape == ref.shape and np.allclose(y64, ref, rtol=1e-12, atol=1e-12)
+    s64, _ = oracle.conv2d(x, w, b, None, ph, pw, alpha=0.75, act=W.ACT_SILU)
+    t = 0.75 * torch.nn.functional.conv2d(xt, wt, None, padding=(ph, pw)) + torch.from_numpy(b.astype(np.float64))[None, :, None, None]
+    assert np.allclose(s64, torch.nn.functional.silu(t).permute(0, 2, 3, 1).numpy(), rtol=1e-12, atol=1e-12)
+
+
+def test_oracle_conv_special_cases(oracle):
+    # 1x1 filter: a plain GEMM over channels -- the (pinned) GEMM oracle with B stored [OC, IC]
+    n, H, Wd, IC, OC = 2, 5, 7, 16, 24
+    x, w, b, r = problem(n, H, Wd, IC, OC, 1, 1, seed=3, residual=True)
+    y64, y16 = oracle.conv2d(x, w, b, r, 0, 0, alpha=0.5, beta=1.0, act=W.ACT_GELU_TANH)
+    g64, g16 = oracle.gemm_epilogue(x.reshape(1, n * H * Wd, IC), w.reshape(1, OC, IC), b, r.reshape(1, n * H * Wd, OC), n * H * Wd, OC, IC, 1,
+                                    0.5, 1.0, W.ACT_GELU_TANH | W.FLAG_B_COLMAJOR)
+    assert np.array_equal(y64.reshape(g64.shape), g64) and np.array_equal(y16.reshape(g16.shape), g16)
+    # a filter with a single 1 at tap (a, b) on the channel diagonal shifts the image; zero padding shows at the border
+    IC = OC = 8
+    x = gen.tensor(4, gen.TENSOR_A, (1, 6, 9, IC), "normal", 1.0)
+    for (a, c) in [(0, 0), (1, 1), (2, 0), (0, 2)]:
+        w = np.zeros((OC, 3, 3, IC), dtype=np.uint16)
+        w[np.arange(OC), a, c, np.arange(IC)] = 0x3F80                        # bf16 1.0
+        y64, y16 = oracle.conv2d(x, w, None, None, 1, 1)
+        want = np.zeros((1, 6, 9, OC))
+        xs = f64(x)
+        for oh in range(6):
+            for ow in range(9):
+                ih, iw = oh + a - 1, ow + c - 1
+                if 0 <= ih < 6 and 0 <= iw < 9:
+                    want[0, oh, ow] = xs[0, ih, iw]
+        assert np.array_equal(y64, want)
+    # all-ones image and filter: every output counts the taps that fall inside the image, times IC
+    x = np.full((1, 5, 6, 8), 0x3F80, dtype=np.uint16)
+    w = np.full((8, 3, 3, 8), 0x3F80, dtype=np.uint16)
+    y64, _ = oracle.conv2d(x, w, None, None, 1, 1)
+    rows = np.array([2, 3, 3, 3, 2])[:, None]
+    cols = np.array([2, 3, 3, 3, 3, 2])[None, :]
+    assert np.array_equal(y64[0, :, :, 0], (rows * cols * 8).astype(np.float64)) and np.all(y64 == y64[..., :1])
+
+
+# ---------------------------------------------------------------- GPU parity
+
+@pytest.fixture(scope="module")
+def ctx():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device")
+    import paper_2604_01489_b200 as cg
+    c = cg.Context(0)
+    yield c
+    c.close()
+
+
+def run_conv(ctx, x, w, b, r, ph, pw, alpha, beta, act):
+    import torch
+    to = lambda a: None if a is None else torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+    n, H, Wd, IC = x.shape
+    OC, KH, KW, _ = w.shape
+    OH, OW = H + 2 * ph - KH + 1, Wd + 2 * pw - KW + 1
+    y = torch.full((n, OH, OW, OC), float("nan"), dtype=torch.bfloat16, device="cuda")
+    bd = None if b is None else torch.from_numpy(b).cuda()
+    ctx.conv2d(to(x), to(w), bd, to(r), y, n, H, Wd, IC, OC, KH, KW, ph, pw, alpha, beta, act)
+    ctx.check()
+    return y.view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+CONV_PLANS = [dict(), dict(tile_n=64, cta_group=1), dict(tile_n=128, cta_group=1), dict(tile_n=256, cta_group=1),
+              dict(tile_n=128, cta_group=2), dict(tile_n=256, cta_group=2), dict(tile_n=512, cta_group=2),
+              dict(tile_n=128, cta_group=1, num_units=13), dict(tile_n=128, cta_group=1, cluster_split=2)]
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("plan", CONV_PLANS, ids=lambda d: "auto" if not d else "-".join(f"{k}{v}" for k, v in d.items()))
+@pytest.mark.parametrize("geom", [(2, 20, 37, 72, 136, 3, 3, 1, 1), (3, 16, 16, 64, 64, 1, 1, 0, 0), (1, 9, 50, 128, 264, 2, 4, 1, 0)], ids=str)
+def test_gpu_conv_integer_operands_bit_exact(ctx, oracle, geom, plan):
+    n, H, Wd, IC, OC, KH, KW, ph, pw = geom
+    x, w, b, r = problem(n, H, Wd, IC, OC, KH, KW, seed=sum(geom), dist=(SI, 1.0), wdist=(SI, 1.0), residual=True, ph=ph, pw=pw)
+    if "cluster_split" in plan and (KH * KW * ((IC + 63) // 64)) % 2:
+        pytest.skip("an odd number of k-blocks cannot be split in two")
+    ctx.set_tuning(reset=True)
+    if plan:
+        ctx.set_tuning(**plan)
+    y = run_conv(ctx, x, w, b, r, ph, pw, 2.0, -1.0, W.ACT_RELU)
+    _, y16 = oracle.conv2d(x, w, b, r, ph, pw, alpha=2.0, beta=-1.0, act=W.ACT_RELU)
+    assert np.array_equal(y, y16), int(np.sum(y != y16))
+    pl = ctx.last_plan()
+    assert pl["k_blocks"] == KH * KW * ((IC + 63) // 64) and pl["latency_kernel"] == 0
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("act", [W.ACT_NONE, W.ACT_GELU_TANH, W.ACT_SILU])
+def test_gpu_conv_random_inputs(ctx, oracle, act):
+    import parity_util as PU
+    n, H, Wd, IC, OC, KH, KW, ph, pw = 2, 30, 45, 96, 200, 3, 3, 1, 1
+    x, w, b, r = problem(n, H, Wd, IC, OC, KH, KW, seed=act + 9, wdist=("normal", 0.05), residual=True, ph=ph, pw=pw)
+    y64, _ = oracle.conv2d(x, w, b, r, ph, pw, alpha=0.7, beta=0.5, act=act)
+    for tuning in (dict(), dict(tile_n=256, cta_group=2)):
+        ctx.set_tuning(reset=True)
+        if tuning:
+            ctx.set_tuning(**tuning)
+        y = run_conv(ctx, x, w, b, r, ph, pw, 0.7, 0.5, act)
+        c = PU.compare(y, y64)
+        assert c["ok"], c
+
+
+@pytest.mark.gpu
+def test_gpu_conv_error_codes(ctx):
+    import torch
+    import paper_2604_01489_b200 as cg
+    x = torch.zeros(1, 8, 8, 8, dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros(8, 3, 3, 8, dtype=torch.bfloat16, device="cuda")
+    y = torch.zeros(1, 6, 6, 8, dtype=torch.bfloat16, device="cuda")
+    h = ctx.handle
+    assert cg.cg_conv2d(h, None, w, None, None, y, 1, 8, 8, 8, 8, 3, 3) == cg.CG_ERR_INVALID_ARG
+    assert cg.cg_conv2d(h, x, w, None, None, y, 1, 8, 8, 8, 8, 9, 3) == cg.CG_ERR_INVALID_ARG       # filter larger than the image
+    assert cg.cg_conv2d(h, x, w, None, None, y, 1, 8, 8, 8, 8, 3, 3, beta=1.0) == cg.CG_ERR_INVALID_ARG
+    assert cg.cg_conv2d(h, x, w, None, None, y, 1, 8, 8, 4, 8, 3, 3) == cg.CG_ERR_UNSUPPORTED       # IC % 8
+    assert cg.cg_conv2d(h, x, w, None, None, y, 1, 8, 8, 8, 8, 3, 3, act=cg.CG_FLAG_B_COLMAJOR) == cg.CG_ERR_INVALID_ARG
+    assert cg.cg_conv2d(h, x, w, None, None, y, 1, 8, 8, 8, 8, 3, 3) == cg.CG_OK
+    ctx.check()
