@@ -205,6 +205,22 @@ int make_map(cg_context* h, CUtensorMap* map, const void* base, uint64_t inner, 
   return CG_OK;
 }
 
+// bf16, rank 4 (channels, width, height, images), dense NHWC, 128-byte swizzle, zero fill outside the tensor.
+int make_map4(cg_context* h, CUtensorMap* map, const void* base, uint64_t c, uint64_t w, uint64_t hh, uint64_t n,
+              uint32_t box_c, uint32_t box_w, uint32_t box_h) {
+  const cuuint64_t dims[4] = {c, w, hh, n};
+  const cuuint64_t strides[3] = {c * 2, c * w * 2, c * w * hh * 2};
+  const cuuint32_t box[4] = {box_c, box_w, box_h, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  const CUresult r = h->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS)
+    return fail(h, CG_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d) for NHWC dims %llu x %llu x %llu x %llu", (int)r,
+                (unsigned long long)n, (unsigned long long)hh, (unsigned long long)w, (unsigned long long)c);
+  return CG_OK;
+}
+
 // ---- plan --------------------------------------------------------------------------
 
 size_t partial_need(long long split_units, int bn, int cgn) {
@@ -429,13 +445,14 @@ int launch_small(cg_context* h, const void* A, const void* B, const void* bias, 
 int grow(cg_context* h, StagingBuf* s, size_t bytes);
 
 int launch(cg_context* h, const void* A, const void* B, const void* bias, const void* R, void* D, int M, int N, int K,
-           int batch, float alpha, float beta, int act, cudaStream_t stream, const cg_epilogue_ex_t* ex = nullptr) {
+           int batch, float alpha, float beta, int act, cudaStream_t stream, const cg_epilogue_ex_t* ex = nullptr,
+           const ConvGeom* conv = nullptr) {
   const bool b_kmajor = (act & CG_FLAG_B_COLMAJOR) != 0;
   const bool ext_in_use = (act & (CG_FLAG_BIAS_PER_ROW | CG_FLAG_B_BROADCAST | CG_FLAG_CLAMP | CG_FLAG_IN_F32)) != 0 ||
                           (ex && (ex->row_scale || ex->col_scale || ex->out_dtype != CG_OUT_BF16 || ex->row_reduce));
   const int row_reduce = ex ? ex->row_reduce : 0;
   const bool store_d = D != nullptr;
-  if (!ext_in_use) {
+  if (!ext_in_use && !conv) {
     const int rs = launch_small(h, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, stream);
     if (rs >= 0) return rs;
   }
@@ -452,18 +469,23 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   lookup(pl.bn, pl.cg, b_kmajor, &e);
 
   CUtensorMap tmA, tmB, tmD, tmR;
-  if ((rc = make_map(h, &tmA, A, K, M, batch, bk_elems, BM, in_dtype)) != CG_OK) return rc;
+  if (conv) rc = make_map4(h, &tmA, A, conv->IC, conv->W, conv->H, conv->n_img, BK, CONV_TILE_W, CONV_TILE_H);
+  else rc = make_map(h, &tmA, A, K, M, batch, bk_elems, BM, in_dtype);
+  if (rc != CG_OK) return rc;
   const int b_entries = b_broadcast ? 1 : batch;
-  if (b_kmajor) rc = make_map(h, &tmB, B, K, N, b_entries, bk_elems, e.sub_cols, in_dtype);
+  if (conv) rc = make_map(h, &tmB, B, static_cast<uint64_t>(conv->KH) * conv->KW * conv->IC, N, 1, BK, e.sub_cols);
+  else if (b_kmajor) rc = make_map(h, &tmB, B, K, N, b_entries, bk_elems, e.sub_cols, in_dtype);
   else rc = make_map(h, &tmB, B, N, K, b_entries, 64, BK);
   if (rc != CG_OK) return rc;
-  if (store_d) rc = make_map(h, &tmD, D, N, M, batch, out_dtype == CG_OUT_F32 ? 32 : EPI_COLS, 32, out_dtype);
+  if (conv) rc = make_map4(h, &tmD, D, N, conv->OW, conv->OH, conv->n_img, EPI_COLS, CONV_TILE_W, 2);
+  else if (store_d) rc = make_map(h, &tmD, D, N, M, batch, out_dtype == CG_OUT_F32 ? 32 : EPI_COLS, 32, out_dtype);
   else rc = make_map(h, &tmD, A, tf32 ? 2 * K : K, M, batch, EPI_COLS, 32);          // never used: any valid 16-bit view
   if (rc != CG_OK) return rc;
   // (unused without a residual)
-  if ((rc = make_map(h, &tmR, beta != 0.0f ? R : (store_d ? D : A), beta != 0.0f || store_d ? N : (tf32 ? 2 * K : K), M, batch,
-                     EPI_COLS, 32)) != CG_OK)
-    return rc;
+  if (conv) rc = make_map4(h, &tmR, beta != 0.0f ? R : D, N, conv->OW, conv->OH, conv->n_img, EPI_COLS, CONV_TILE_W, 2);
+  else rc = make_map(h, &tmR, beta != 0.0f ? R : (store_d ? D : A), beta != 0.0f || store_d ? N : (tf32 ? 2 * K : K), M, batch,
+                     EPI_COLS, 32);
+  if (rc != CG_OK) return rc;
 
   KernelParams p;
   memset(&p, 0, sizeof p);
@@ -496,6 +518,7 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   p.clamp = (act & CG_FLAG_CLAMP) ? 1 : 0;
   p.out_dtype = out_dtype;
   p.tf32 = tf32 ? 1 : 0;
+  if (conv) p.cv = *conv;
   if (ex) {
     p.clamp_lo = ex->clamp_lo;
     p.clamp_hi = ex->clamp_hi;
@@ -654,6 +677,36 @@ int cg_gemm_epilogue_ex(cg_handle_t h, const void* A, const void* B, const void*
     return fail(h, CG_ERR_INVALID_ARG, "CG_FLAG_CLAMP needs the bounds of a cg_epilogue_ex_t");
   }
   return launch(h, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, static_cast<cudaStream_t>(stream), ex);
+}
+
+int cg_conv2d(cg_handle_t h, const void* x, const void* w, const void* bias, const void* R, void* y, int n_img, int H, int W,
+              int IC, int OC, int KH, int KW, int pad_h, int pad_w, float alpha, float beta, int act, void* stream) {
+  if (!h) return CG_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(h->mu);
+  if (!x || !w || !y) return fail(h, CG_ERR_INVALID_ARG, "x, w and y must not be NULL");
+  if (n_img < 1 || H < 1 || W < 1 || IC < 1 || OC < 1 || KH < 1 || KW < 1 || pad_h < 0 || pad_w < 0)
+    return fail(h, CG_ERR_INVALID_ARG, "sizes must be >= 1 and paddings >= 0");
+  const int OH = H + 2 * pad_h - KH + 1, OW = W + 2 * pad_w - KW + 1;
+  if (OH < 1 || OW < 1) return fail(h, CG_ERR_INVALID_ARG, "the filter does not fit the padded image");
+  const int kind = act & 0xFF;
+  if (kind > CG_ACT_LEAKY_RELU || (act & ~(0xFF | CG_FLAG_BIAS_BF16)) != 0 || act < 0)
+    return fail(h, CG_ERR_INVALID_ARG, "unknown activation or flag bits in act=0x%x", act);
+  if (beta != 0.0f && !R) return fail(h, CG_ERR_INVALID_ARG, "R must not be NULL when beta != 0");
+  if (IC % 8 != 0 || OC % 8 != 0) return fail(h, CG_ERR_UNSUPPORTED, "IC and OC must be multiples of 8 (got %d, %d)", IC, OC);
+  int rc = check_alignment(h, x, w, bias, R, y, beta, act);
+  if (rc != CG_OK) return rc;
+  ConvGeom g;
+  memset(&g, 0, sizeof g);
+  g.on = 1; g.n_img = n_img; g.H = H; g.W = W; g.OH = OH; g.OW = OW; g.KH = KH; g.KW = KW; g.pad_h = pad_h; g.pad_w = pad_w; g.IC = IC;
+  g.ic_blocks = ceil_div(IC, BK);
+  g.tiles_h = ceil_div(OH, CONV_TILE_H);
+  g.tiles_w = ceil_div(OW, CONV_TILE_W);
+  const long long pixel_tiles = static_cast<long long>(n_img) * g.tiles_h * g.tiles_w;
+  const long long k_blocks = static_cast<long long>(KH) * KW * g.ic_blocks;
+  if (pixel_tiles * BM >= (1ll << 30) || k_blocks * BK >= (1ll << 30)) return fail(h, CG_ERR_UNSUPPORTED, "convolution too large");
+  // the GEMM the kernel sees: rows = padded pixel tiles, columns = output channels, K = taps x channel blocks
+  return launch(h, x, w, bias, R, y, static_cast<int>(pixel_tiles * BM), OC, static_cast<int>(k_blocks * BK), 1, alpha, beta,
+                act | CG_FLAG_B_COLMAJOR, static_cast<cudaStream_t>(stream), nullptr, &g);
 }
 
 int cg_diag_matmul(cg_handle_t h, const float* d, const void* B, void* C, long long M, int N, int dtype, void* stream) {

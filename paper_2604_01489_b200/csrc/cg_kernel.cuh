@@ -74,6 +74,18 @@ enum { OUT_BF16 = 0, OUT_F16 = 1, OUT_F32 = 2 };
 enum { REDUCE_NONE = 0, REDUCE_SUM = 1, REDUCE_MAX = 2, REDUCE_LOGSUMEXP = 3 };
 enum { STATUS_OK = 0, STATUS_SMEM = 4, STATUS_TIMEOUT = 6 };
 
+// Implicit-GEMM convolution (stride 1, NHWC): output pixels are the GEMM's rows, in tiles of 8 x 16
+// pixels (128 rows); output channels its columns; K runs over (kh, kw, 64-channel block).  A k-block of
+// the A operand is one rank-4 TMA box of the input -- 64 channels x 16 x 8 pixels, shifted by the tap
+// and the padding; whatever falls outside the image is zero-filled by the TMA unit, which is the padding.
+struct ConvGeom {
+  int on;
+  int n_img, H, W, OH, OW, KH, KW, pad_h, pad_w, IC;
+  int ic_blocks;          // ceil(IC / 64)
+  int tiles_h, tiles_w;   // pixel tiles per image
+};
+constexpr int CONV_TILE_H = 8, CONV_TILE_W = 16;
+
 struct KernelParams {
   int M, N, K, batch;
   int tiles_m, tiles_n;   // tiles per batch entry; a tile is (CG*128) x BN
@@ -105,6 +117,7 @@ struct KernelParams {
   int store_d;            // 0: D is not wanted, only the row reduction
   int row_slots;          // partial results per row: tiles_n x K parts of a cluster x column groups
   float* row_ws;          // [batch*M][row_slots] (two floats per slot for logsumexp: running maximum, scaled sum)
+  ConvGeom cv;            // cv.on: A is an NHWC image read through a rank-4 map, D (and R) NHWC through rank-4 maps
   int tf32;               // A and B are fp32 and multiplied as TF32: a k-block is 32 elements (still 128 bytes),
                           // one MMA covers 8 of them; B is K-major
   float clamp_lo, clamp_hi;
@@ -248,6 +261,18 @@ __device__ __forceinline__ void trace_event(const KernelParams& p, int ev) {
     p.trace[blockIdx.x * TR_SLOTS + ev] = t;
     if (ev == TR_START || ev == TR_END) p.trace[blockIdx.x * TR_SLOTS + (ev == TR_START ? TR_CLOCK_START : TR_CLOCK_END)] = clock64();
   }
+}
+
+// Virtual row (pixel tile * 128 + row in tile, a multiple of 32) -> image, first output row, first output column
+// of the 2 x 16 pixel strip those 32 rows are.
+__device__ __forceinline__ void conv_strip(const KernelParams& p, int row0, int& n, int& h, int& w) {
+  const int pt = row0 >> 7, sub = (row0 & 127) >> 5;
+  const int per_img = p.cv.tiles_h * p.cv.tiles_w;
+  n = pt / per_img;
+  const int r = pt - n * per_img;
+  const int th = r / p.cv.tiles_w;
+  h = th * CONV_TILE_H + sub * 2;
+  w = (r - th * p.cv.tiles_w) * CONV_TILE_W;
 }
 
 // Bounded mbarrier wait.  false: gave up (limit expired here, or another role aborted).
@@ -409,9 +434,18 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     const uint32_t bar = ptx::smem_u32(&ctrl->full[stage]);
     const uint32_t a_dst = ring_addr + stage * C::STAGE_BYTES;
     const uint32_t b_dst = a_dst + C::A_BYTES;
-    const int k0 = kb * (p.tf32 ? BK / 2 : BK);        // element coordinate: 128 bytes of K per block either way
+    int k0 = kb * (p.tf32 ? BK / 2 : BK);              // element coordinate: 128 bytes of K per block either way
     ptx::mbar_arrive_expect_tx(bar, C::STAGE_BYTES);
-    if (!withhold_a) ptx::tma_load_3d(a_dst, &tmA, bar, k0, m0, b);     // (withheld only by the starvation test hook)
+    if (p.cv.on) {
+      const int tap = kb / p.cv.ic_blocks, icb = kb - tap * p.cv.ic_blocks;
+      const int kh = tap / p.cv.KW, kw = tap - kh * p.cv.KW;
+      int n, h0, w0;
+      conv_strip(p, m0, n, h0, w0);
+      if (!withhold_a) ptx::tma_load_4d(a_dst, &tmA, bar, icb * BK, w0 - p.cv.pad_w + kw, h0 - p.cv.pad_h + kh, n);
+      k0 = tap * p.cv.IC + icb * BK;                   // the weights' K index of this block
+    } else if (!withhold_a) {
+      ptx::tma_load_3d(a_dst, &tmA, bar, k0, m0, b);   // (withheld only by the starvation test hook)
+    }
 #pragma unroll
     for (int h = 0; h < C::NSUB; ++h) {
       const int nh = n0 + h * C::MMA_N;
@@ -482,14 +516,23 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           if (!wait_bar(empty0 + stage * 8, phase ^ 1u, ctrl, p)) { ok = false; break; }
           const uint32_t a_dst = ring_addr + stage * C::STAGE_BYTES;
           const uint32_t b_dst = a_dst + C::A_BYTES;
-          const int k0 = kb * (p.tf32 ? BK / 2 : BK);
+          int k0 = kb * (p.tf32 ? BK / 2 : BK);
           if constexpr (CG == 1) {
             issue_loads(stage, kb, m0, n0, b, bb, p.test_starve && issued == 0);
           } else {
             // both CTAs' bytes are counted on the leader's barrier
             if (cta_rank == 0) ptx::mbar_arrive_expect_tx(full0 + stage * 8, 2 * C::STAGE_BYTES);
             const uint32_t bar = full0_leader + stage * 8;
-            if (!(p.test_starve && issued == 0)) ptx::tma_load_3d_pair(a_dst, &tmA, bar, k0, m0, b);
+            if (p.cv.on) {
+              const int tap = kb / p.cv.ic_blocks, icb = kb - tap * p.cv.ic_blocks;
+              const int kh = tap / p.cv.KW, kw = tap - kh * p.cv.KW;
+              int n, h0, w0;
+              conv_strip(p, m0, n, h0, w0);
+              ptx::tma_load_4d_pair(a_dst, &tmA, bar, icb * BK, w0 - p.cv.pad_w + kw, h0 - p.cv.pad_h + kh, n);
+              k0 = tap * p.cv.IC + icb * BK;
+            } else if (!(p.test_starve && issued == 0)) {
+              ptx::tma_load_3d_pair(a_dst, &tmA, bar, k0, m0, b);
+            }
 #pragma unroll
             for (int h = 0; h < C::NSUB; ++h) {
               const int nh = n0 + h * C::MMA_N;
@@ -660,7 +703,13 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           dst = stage_base + store_buf * EPI_BUF_BYTES;
         }
         ptx::mbar_arrive_expect_tx(r_bar, EPI_BUF_BYTES);
-        ptx::tma_load_3d(dst, &tmR, r_bar, col, row0, bb);      // outside the tensor: zero fill, same byte count
+        if (p.cv.on) {
+          int n, h, w;
+          conv_strip(p, row0, n, h, w);
+          ptx::tma_load_4d(dst, &tmR, r_bar, col, w, h, n);
+        } else {
+          ptx::tma_load_3d(dst, &tmR, r_bar, col, row0, bb);    // outside the tensor: zero fill, same byte count
+        }
       }
       r_pending = true;
     };
@@ -678,6 +727,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     };
     // Pulls this thread's row of a tile's residual (its share of the columns) into L2.
     auto prefetch_residual = [&](const Segment& sg) {
+      if (p.cv.on) return;               // (rows are not contiguous pixels there)
       int pb, pmt, pnt;
       decode_tile(p, sg.tile, pb, pmt, pnt);
       const int pm = pmt * (BM * CG) + static_cast<int>(cta_rank) * BM + row_in_tile;
@@ -719,7 +769,12 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       decode_tile(p, s.tile, b, mt, nt);
       const int m_base = mt * (BM * CG) + static_cast<int>(cta_rank) * BM;   // first row of this CTA's slab
       const int n_base = nt * BN;
-      const bool warp_rows_valid = (m_base + q * 32) < p.M;
+      bool warp_rows_valid = (m_base + q * 32) < p.M;
+      int cv_n = 0, cv_h = 0, cv_w = 0;                 // convolution: this warp's 2 x 16 strip of output pixels
+      if (p.cv.on) {
+        conv_strip(p, m_base + q * 32, cv_n, cv_h, cv_w);
+        warp_rows_valid = cv_n < p.cv.n_img && cv_h < p.cv.OH;
+      }
       const bool whole_tile = (s.kb0 == 0 && s.kb1 == p.k_blocks);
       int n_chunks = (p.N - n_base + EPI_COLS - 1) / EPI_COLS;    // chunks with at least one valid column
       if (n_chunks > BN / EPI_COLS) n_chunks = BN / EPI_COLS;
@@ -1028,7 +1083,10 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           __syncwarp();
           if (!dry && ew == 0 && lane == 0 && c == c_lo) trace_event(p, TR_EPI_STAGED);
           if (lane == 0) {
-            if (warp_rows_valid && !dry) ptx::tma_store_3d(&tmD, buf_addr, n0, m_base + q * 32, b);   // clips rows >= M, cols >= N
+            if (warp_rows_valid && !dry) {
+            if (p.cv.on) ptx::tma_store_4d(&tmD, buf_addr, n0, cv_w, cv_h, cv_n);                   // clips pixels outside the image
+            else ptx::tma_store_3d(&tmD, buf_addr, n0, m_base + q * 32, b);                          // clips rows >= M, cols >= N
+          }
             ptx::bulk_commit_group();
             if (ew == 0 && !dry) trace_event(p, c == c_lo ? TR_FIRST_STORE : TR_LAST_STORE);
           }
