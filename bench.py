@@ -430,6 +430,41 @@ def diag_rows(ctx, device, peaks, flush):
     return out
 
 
+def conv_row(ctx, device, peaks, flush):
+    """3x3 convolution + bias + ReLU as an implicit GEMM: 16 images of 64 x 64 x 256 channels -> 256 channels,
+    padding 1 (77.3 GFLOP); PyTorch's channels-last convolution (library kernel) + bias + ReLU alongside."""
+    import torch
+    import torch.nn.functional as F
+    n, H, Wd, IC, OC, KH, KW, pad = 16, 64, 64, 256, 256, 3, 3, 1
+    g = torch.Generator(device=device)
+    g.manual_seed(6)
+    x = torch.randn((n, H, Wd, IC), device=device, generator=g).to(torch.bfloat16)
+    w = (torch.randn((OC, KH, KW, IC), device=device, generator=g) * 0.02).to(torch.bfloat16)
+    bias = torch.randn((OC,), device=device, generator=g)
+    y = torch.empty((n, H, Wd, OC), device=device, dtype=torch.bfloat16)
+    call = lambda: ctx.conv2d(x, w, bias, None, y, n, H, Wd, IC, OC, KH, KW, pad, pad, 1.0, 0.0, W.ACT_RELU)
+    timed(call, 3, flush)
+    ts = timed(call, 10, flush)
+    ctx.check()
+    plan = ctx.last_plan()
+    xc = x.permute(0, 3, 1, 2)                          # NCHW views of the channels-last tensors
+    wc = w.permute(0, 3, 1, 2)
+    bb = bias.to(torch.bfloat16)
+    lib = lambda: torch.relu(F.conv2d(xc, wc, bb, padding=pad))
+    lib_only = lambda: F.conv2d(xc, wc, None, padding=pad)
+    timed(lib, 3, flush)
+    tl = timed(lib, 10, flush)
+    timed(lib_only, 3, flush)
+    tlo = timed(lib_only, 10, flush)
+    flops = 2.0 * n * H * Wd * OC * IC * KH * KW
+    best = min(ts)
+    nbytes = 2 * (x.numel() + w.numel() + y.numel()) + 4 * OC
+    return {"workload": "conv 3x3 pad 1, 16 x 64 x 64 x 256 -> 256 channels, NHWC bf16, bias fp32, ReLU", "flops": flops,
+            "us_best": best * 1e6, "us_median": float(np.median(ts)) * 1e6, "tflops_best": flops / best / 1e12,
+            "frac_tensor_of_measured_burst": flops / best / 1e12 / peaks["bf16_tflops"], "algorithmic_bytes": nbytes,
+            "torch_conv_bias_relu_us_best": min(tl) * 1e6, "torch_conv_only_us_best": min(tlo) * 1e6, "plan": plan}
+
+
 def workload_table(ctx, device, peaks, names):
     """All five workloads under the heuristic plan, each launch timed alone after an L2 flush (their
     inputs may fit in L2)."""
@@ -462,6 +497,7 @@ def workload_table(ctx, device, peaks, names):
         ctx.set_tuning(reset=True)
         out["next_tf32_8192"] = tf32_row(ctx, device, peaks, flush)
         out["next_diag_matmul_8192"] = diag_rows(ctx, device, peaks, flush)
+        out["next_conv3x3_256"] = conv_row(ctx, device, peaks, flush)
     return out
 
 
@@ -593,7 +629,8 @@ def run_row(args):
     device = torch.device("cuda", 0)
     ctx = cg.Context(0)
     flush = L2Flush(device)
-    row = tf32_row(ctx, device, load_peaks(), flush) if args.row == "tf32" else diag_rows(ctx, device, load_peaks(), flush)
+    fn = {"tf32": tf32_row, "diag": diag_rows, "conv": conv_row}[args.row]
+    row = fn(ctx, device, load_peaks(), flush)
     print(json.dumps({"row": args.row, "result": row}), flush=True)
 
 
@@ -607,7 +644,7 @@ def main():
     ap.add_argument("--no-table", action="store_true", help="skip the five-workload table")
     for flag in ("tile-n", "cta-group", "num-units", "dp-units", "stages", "group-m", "max-ctas"):
         ap.add_argument(f"--{flag}", type=int, default=0, help="plan override for ablations (0 = heuristic)")
-    ap.add_argument("--row", choices=["tf32", "diag"], default=None,
+    ap.add_argument("--row", choices=["tf32", "diag", "conv"], default=None,
                     help="only that row of the 'next' part of the table (a few launches; for profiler runs)")
     ap.add_argument("--kernel-only", action="store_true",
                     help="only the device-timed region (for profiler runs): no e2e, no CPU baseline, no table")
