@@ -8,8 +8,10 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcg.so")
-SOURCES = ["cg_api.cu"]
-HEADERS = ["cg_kernel.cuh", "cg_ptx.cuh", os.path.join("..", "..", "include", "cg.h")]
+SOURCES = ["cg_api.cu", "cg_inst.cu"]
+HEADERS = ["cg_kernel.cuh", "cg_small.cuh", "cg_diag.cuh", "cg_reduce.cuh", "cg_instances.h", "cg_ptx.cuh", os.path.join("..", "..", "include", "cg.h")]
+INSTANCE_GROUPS = 6          # cg_inst.cu is compiled once per group of kernel instances, in parallel
+OBJ_DIR = os.path.join(HERE, "build")
 
 
 def _nvcc() -> str:
@@ -30,17 +32,32 @@ def stale() -> bool:
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not stale():
         return LIB
-    cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "-Xcompiler", "-fPIC,-fvisibility=hidden", "-shared", "-o", LIB]
+    from concurrent.futures import ThreadPoolExecutor
+    os.makedirs(OBJ_DIR, exist_ok=True)
+    flags = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC,-fvisibility=hidden"]
     if verbose:
-        cmd += ["-Xptxas", "-v"]
-    cmd += [os.path.join(CSRC, s) for s in SOURCES]
-    cmd += ["-lcudart"]
-    res = subprocess.run(cmd, capture_output=True, text=True)
-    if verbose or res.returncode != 0:
-        sys.stderr.write(res.stdout + res.stderr)
-    if res.returncode != 0:
-        raise RuntimeError("nvcc failed building libcg.so")
+        flags += ["-Xptxas", "-v"]
+    jobs = [(os.path.join(CSRC, "cg_api.cu"), os.path.join(OBJ_DIR, "cg_api.o"), [])]
+    jobs += [(os.path.join(CSRC, "cg_inst.cu"), os.path.join(OBJ_DIR, f"cg_inst_{g}.o"), [f"-DCG_INST_GROUP={g}"])
+             for g in range(INSTANCE_GROUPS)]
+
+    def compile_one(job):
+        src, obj, extra = job
+        return subprocess.run([_nvcc()] + flags + extra + ["-c", src, "-o", obj], capture_output=True, text=True)
+
+    with ThreadPoolExecutor(max_workers=min(len(jobs), os.cpu_count() or 1)) as pool:
+        results = list(pool.map(compile_one, jobs))
+    for res in results:
+        if verbose or res.returncode != 0:
+            sys.stderr.write(res.stdout + res.stderr)
+    if any(r.returncode != 0 for r in results):
+        raise RuntimeError("nvcc failed compiling libcg.so")
+    link = subprocess.run([_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", LIB] + [j[1] for j in jobs] + ["-lcudart"],
+                          capture_output=True, text=True)
+    if verbose or link.returncode != 0:
+        sys.stderr.write(link.stdout + link.stderr)
+    if link.returncode != 0:
+        raise RuntimeError("nvcc failed linking libcg.so")
     return LIB
 
 

@@ -14,8 +14,17 @@
 #include <mutex>
 
 #include "cg_kernel.cuh"
+#include "cg_instances.h"
 #include "cg_small.cuh"
+#include "cg_reduce.cuh"
 #include "cg_diag.cuh"
+
+namespace cg {
+// the kernel instances are compiled in translation units of their own (cg_inst.cu)
+#define CG_DECLARE(BN, CGN, KM, CV) extern template CG_KERNEL_SIGNATURE(BN, CGN, KM, CV)
+CG_ALL_INSTANCES(CG_DECLARE)
+#undef CG_DECLARE
+}  // namespace cg
 
 namespace {
 
@@ -121,15 +130,24 @@ struct KernelEntry {
   int stage_bytes, fixed_bytes, r_bytes, stages_max, stages_max_r, threads, sub_cols;
 };
 
-template <int BN, int CGN, bool KM>
+template <int BN, int CGN, bool KM, bool CONV = false>
 KernelEntry entry() {
   using C = Cfg<BN, CGN, KM>;
-  return KernelEntry{gemm_epilogue_kernel<BN, CGN, KM>, C::STAGE_BYTES, C::FIXED_BYTES, C::R_BYTES, C::stages_max(false),
+  return KernelEntry{gemm_epilogue_kernel<BN, CGN, KM, CONV>, C::STAGE_BYTES, C::FIXED_BYTES, C::R_BYTES, C::stages_max(false),
                      C::stages_max(true), C::NUM_THREADS, C::SUB_COLS};
 }
 
 // index: [bn_idx (64,128,256)][cg-1][b_kmajor]
-bool lookup(int bn, int cgn, bool km, KernelEntry* out) {
+bool lookup(int bn, int cgn, bool km, KernelEntry* out, bool conv = false) {
+  if (conv) {                 // the convolution instances: K-major weights, rank-4 maps for the image and the output
+    if (cgn == 1 && bn == 64) { *out = entry<64, 1, true, true>(); return true; }
+    if (cgn == 1 && bn == 128) { *out = entry<128, 1, true, true>(); return true; }
+    if (cgn == 1 && bn == 256) { *out = entry<256, 1, true, true>(); return true; }
+    if (cgn == 2 && bn == 128) { *out = entry<128, 2, true, true>(); return true; }
+    if (cgn == 2 && bn == 256) { *out = entry<256, 2, true, true>(); return true; }
+    if (cgn == 2 && bn == 512) { *out = entry<512, 2, true, true>(); return true; }
+    return false;
+  }
   if (cgn == 1) {
     if (bn == 64) { *out = km ? entry<64, 1, true>() : entry<64, 1, false>(); return true; }
     if (bn == 128) { *out = km ? entry<128, 1, true>() : entry<128, 1, false>(); return true; }
@@ -165,6 +183,9 @@ int prepare_kernels(cg_context* h) {
         if (!lookup(bns[i], cgn, km != 0, &e)) continue;
         CG_CUDA(h, cudaFuncSetAttribute(reinterpret_cast<const void*>(e.fn), cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         SMEM_LIMIT));
+        if (km != 0 && lookup(bns[i], cgn, true, &e, true))
+          CG_CUDA(h, cudaFuncSetAttribute(reinterpret_cast<const void*>(e.fn), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          SMEM_LIMIT));
       }
   for (int act = 0; act <= CG_ACT_LEAKY_RELU; ++act)
     CG_CUDA(h, cudaFuncSetAttribute(reinterpret_cast<const void*>(small_kernel_for(act)), cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -466,7 +487,7 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   int rc = make_plan(h, M, N, K, batch, b_kmajor, beta != 0.0f, &pl, out_dtype == CG_OUT_F32 || !store_d, bk_elems);
   if (rc != CG_OK) return rc;
   KernelEntry e;
-  lookup(pl.bn, pl.cg, b_kmajor, &e);
+  lookup(pl.bn, pl.cg, b_kmajor, &e, conv != nullptr);
 
   CUtensorMap tmA, tmB, tmD, tmR;
   if (conv) rc = make_map4(h, &tmA, A, conv->IC, conv->W, conv->H, conv->n_img, BK, CONV_TILE_W, CONV_TILE_H);

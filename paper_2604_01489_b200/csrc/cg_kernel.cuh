@@ -395,7 +395,7 @@ __device__ __forceinline__ void stage_chunk(const uint32_t (&out)[EPI_COLS / 2],
 
 // ---------------------------------------------------------------- the kernel
 
-template <int BN, int CG, bool B_KMAJOR>
+template <int BN, int CG, bool B_KMAJOR, bool CONV = false>
 __global__ void __launch_bounds__((Cfg<BN, CG, B_KMAJOR>::NUM_THREADS), 1)
 gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                      const __grid_constant__ CUtensorMap tmD, const __grid_constant__ CUtensorMap tmR,
@@ -436,7 +436,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     const uint32_t b_dst = a_dst + C::A_BYTES;
     int k0 = kb * (p.tf32 ? BK / 2 : BK);              // element coordinate: 128 bytes of K per block either way
     ptx::mbar_arrive_expect_tx(bar, C::STAGE_BYTES);
-    if (p.cv.on) {
+    if constexpr (CONV) {
       const int tap = kb / p.cv.ic_blocks, icb = kb - tap * p.cv.ic_blocks;
       const int kh = tap / p.cv.KW, kw = tap - kh * p.cv.KW;
       int n, h0, w0;
@@ -523,7 +523,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             // both CTAs' bytes are counted on the leader's barrier
             if (cta_rank == 0) ptx::mbar_arrive_expect_tx(full0 + stage * 8, 2 * C::STAGE_BYTES);
             const uint32_t bar = full0_leader + stage * 8;
-            if (p.cv.on) {
+            if constexpr (CONV) {
               const int tap = kb / p.cv.ic_blocks, icb = kb - tap * p.cv.ic_blocks;
               const int kh = tap / p.cv.KW, kw = tap - kh * p.cv.KW;
               int n, h0, w0;
@@ -703,7 +703,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           dst = stage_base + store_buf * EPI_BUF_BYTES;
         }
         ptx::mbar_arrive_expect_tx(r_bar, EPI_BUF_BYTES);
-        if (p.cv.on) {
+        if constexpr (CONV) {
           int n, h, w;
           conv_strip(p, row0, n, h, w);
           ptx::tma_load_4d(dst, &tmR, r_bar, col, w, h, n);
@@ -727,7 +727,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     };
     // Pulls this thread's row of a tile's residual (its share of the columns) into L2.
     auto prefetch_residual = [&](const Segment& sg) {
-      if (p.cv.on) return;               // (rows are not contiguous pixels there)
+      if constexpr (CONV) return;               // (rows are not contiguous pixels there)
       int pb, pmt, pnt;
       decode_tile(p, sg.tile, pb, pmt, pnt);
       const int pm = pmt * (BM * CG) + static_cast<int>(cta_rank) * BM + row_in_tile;
@@ -771,7 +771,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       const int n_base = nt * BN;
       bool warp_rows_valid = (m_base + q * 32) < p.M;
       int cv_n = 0, cv_h = 0, cv_w = 0;                 // convolution: this warp's 2 x 16 strip of output pixels
-      if (p.cv.on) {
+      if constexpr (CONV) {
         conv_strip(p, m_base + q * 32, cv_n, cv_h, cv_w);
         warp_rows_valid = cv_n < p.cv.n_img && cv_h < p.cv.OH;
       }
@@ -1084,7 +1084,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           if (!dry && ew == 0 && lane == 0 && c == c_lo) trace_event(p, TR_EPI_STAGED);
           if (lane == 0) {
             if (warp_rows_valid && !dry) {
-            if (p.cv.on) ptx::tma_store_4d(&tmD, buf_addr, n0, cv_w, cv_h, cv_n);                   // clips pixels outside the image
+            if constexpr (CONV) ptx::tma_store_4d(&tmD, buf_addr, n0, cv_w, cv_h, cv_n);                   // clips pixels outside the image
             else ptx::tma_store_3d(&tmD, buf_addr, n0, m_base + q * 32, b);                          // clips rows >= M, cols >= N
           }
             ptx::bulk_commit_group();
@@ -1146,26 +1146,6 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     ptx::tc_fence_after();
     ptx::tmem_dealloc<CG>(tmem_base, C::TMEM_COLS);
     if (lane == 0) trace_event(p, TR_END);
-  }
-}
-
-// Second pass of the fused row reduction: one thread per row combines its row's partials in slot order.
-__global__ void row_finalize_kernel(const float* __restrict__ ws, float* __restrict__ out, long long rows, int slots, int op) {
-  const long long row = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
-  if (row >= rows) return;
-  if (op == REDUCE_LOGSUMEXP) {
-    const float2* w = reinterpret_cast<const float2*>(ws) + row * slots;
-    float mx = -INFINITY;
-    for (int s = 0; s < slots; ++s) mx = fmaxf(mx, w[s].x);
-    float sum = 0.0f;
-    for (int s = 0; s < slots; ++s)
-      if (w[s].x > -INFINITY) sum += w[s].y * expf(w[s].x - mx);
-    out[row] = mx + logf(sum);
-  } else {
-    const float* w = ws + row * slots;
-    float acc = op == REDUCE_SUM ? 0.0f : -INFINITY;
-    for (int s = 0; s < slots; ++s) acc = op == REDUCE_SUM ? acc + w[s] : fmaxf(acc, w[s]);
-    out[row] = acc;
   }
 }
 
