@@ -144,20 +144,22 @@ CG_API int cg_gemm_epilogue_ex(cg_handle_t h, const void* A, const void* B, cons
  * "convolution followed by bias addition and an activation"; its conv guidance maps M = output channels,
  * N = output pixels, K = IC*KH*KW -- here pixels are the rows and channels the columns, the transpose):
  *
- *   y[n,oh,ow,oc] = act( alpha * sum_{kh,kw,ic} x[n, oh+kh-pad_h, ow+kw-pad_w, ic] * w[oc,kh,kw,ic] + bias[oc] )
- *                   + beta * R[n,oh,ow,oc]            (x is zero outside the image)
+ *   y[n,oh,ow,oc] = act( alpha * sum_{kh,kw,ic} x[n, oh*stride + kh*dilation - pad_h, ow*stride + kw*dilation - pad_w, ic]
+ *                                              * w[oc,kh,kw,ic] + bias[oc] ) + beta * R[n,oh,ow,oc]     (x is zero outside the image)
  *
  *   x     device, bf16 NHWC [n_img,H,W,IC];   w  device, bf16 [OC,KH,KW,IC];   bias fp32/bf16 [OC] or NULL
- *   R, y  device, bf16 NHWC [n_img,OH,OW,OC] with OH = H + 2*pad_h - KH + 1, OW = W + 2*pad_w - KW + 1; R may alias y
- *   stride 1, dilation 1; IC % 8 == 0 and OC % 8 == 0; all tensors dense and 16-byte aligned;
+ *   R, y  device, bf16 NHWC [n_img,OH,OW,OC] with OH = (H + 2*pad_h - (KH-1)*dilation - 1) / stride + 1, OW likewise;
+ *         R may alias y
+ *   stride 1..8 and dilation >= 1, the same in both directions; IC % 8 == 0 and OC % 8 == 0; all tensors dense and
+ *   16-byte aligned;
  *   act: activation | CG_FLAG_BIAS_BF16.
- * No im2col buffer exists anywhere: the producer reads 64-channel x 16 x 8-pixel boxes of x, shifted by the
- * tap, straight into the operand ring; the padding is the TMA unit's zero fill.  Same plans (pair tiles,
+ * No im2col buffer exists anywhere: the producer reads 64-channel x 16 x 8-pixel boxes of x, (every stride-th
+ * pixel, through the box's traversal stride), shifted by the tap, straight into the operand ring; the padding is the TMA unit's zero fill.  Same plans (pair tiles,
  * split-K, cluster split), same errors as cg_gemm_epilogue.
  */
 CG_API int cg_conv2d(cg_handle_t h, const void* x, const void* w, const void* bias, const void* R, void* y, int n_img,
-                     int H, int W, int IC, int OC, int KH, int KW, int pad_h, int pad_w, float alpha, float beta, int act,
-                     void* stream);
+                     int H, int W, int IC, int OC, int KH, int KW, int pad_h, int pad_w, int stride, int dilation,
+                     float alpha, float beta, int act, void* stream);
 
 /*
  * Structured matmul C = diag(d) * B, i.e. C[i,j] = d[i] * B[i,j]: the paper's example of a product whose

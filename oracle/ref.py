@@ -77,7 +77,7 @@ def _load():
         lib.cg_ref_gemm_epilogue_reduce.argtypes = [vp, vp, vp, vp, vp, i64, vp, vp, vp, ci, i64, i64, i64, i64, dbl, dbl, ci, vp, vp,
                                                     dbl, dbl, ci]
         lib.cg_ref_gemm_epilogue_reduce.restype = ci
-        lib.cg_ref_conv2d.argtypes = [vp, vp, vp, vp, vp, vp] + [i64] * 9 + [dbl, dbl, ci]
+        lib.cg_ref_conv2d.argtypes = [vp, vp, vp, vp, vp, vp] + [i64] * 11 + [dbl, dbl, ci]
         lib.cg_ref_conv2d.restype = ci
         lib.cg_ref_diag_matmul.argtypes = [vp, vp, vp, vp, i64, i64, ci]
         lib.cg_ref_diag_matmul.restype = ci
@@ -206,8 +206,8 @@ def gemm_epilogue_reduce(A, B, bias, R, M, N, K, batch, alpha, beta, act, reduce
     return d64, dout, red
 
 
-def conv2d(x, w, bias, R, pad_h, pad_w, alpha=1.0, beta=0.0, act=ACT_NONE):
-    """Stride-1 NHWC convolution with the fused epilogue.  x [n,H,W,IC], w [OC,KH,KW,IC], R [n,OH,OW,OC]: uint16 bf16
+def conv2d(x, w, bias, R, pad_h, pad_w, alpha=1.0, beta=0.0, act=ACT_NONE, stride=1, dilation=1):
+    """NHWC convolution (zero padding, one stride and dilation for both directions) with the fused epilogue.  x [n,H,W,IC], w [OC,KH,KW,IC], R [n,OH,OW,OC]: uint16 bf16
     bits; bias float32 (uint16 with FLAG_BIAS_BF16) [OC].  Returns (Y64, Ybf16 bits) of shape [n,OH,OW,OC]."""
     for name, a in (("x", x), ("w", w)):
         if a.dtype != np.uint16 or a.ndim != 4 or not a.flags.c_contiguous:
@@ -216,11 +216,11 @@ def conv2d(x, w, bias, R, pad_h, pad_w, alpha=1.0, beta=0.0, act=ACT_NONE):
     OC, KH, KW, IC2 = w.shape
     if IC2 != IC:
         raise ValueError("channel counts differ")
-    OH, OW = H + 2 * pad_h - KH + 1, W + 2 * pad_w - KW + 1
+    OH, OW = (H + 2 * pad_h - (KH - 1) * dilation - 1) // stride + 1, (W + 2 * pad_w - (KW - 1) * dilation - 1) // stride + 1
     y64 = np.empty((n, OH, OW, OC), dtype=np.float64)
     y16 = np.empty((n, OH, OW, OC), dtype=np.uint16)
     rc = _load().cg_ref_conv2d(_ptr(x), _ptr(w), _ptr(bias), _ptr(R), _ptr(y64), _ptr(y16), n, H, W, IC, OC, KH, KW, pad_h, pad_w,
-                               float(alpha), float(beta), int(act))
+                               int(stride), int(dilation), float(alpha), float(beta), int(act))
     if rc != 0:
         raise ValueError("oracle rejected the arguments")
     return y64, y16

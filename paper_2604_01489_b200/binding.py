@@ -78,7 +78,7 @@ def load() -> ctypes.CDLL:
     lib.cg_gemm_epilogue.argtypes = gemm_args
     lib.cg_gemm_epilogue_host.argtypes = gemm_args
     lib.cg_gemm_epilogue_ex.argtypes = gemm_args[:-1] + [ctypes.POINTER(cg_epilogue_ex_t), vp]
-    lib.cg_conv2d.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, cf, cf, ci, vp]
+    lib.cg_conv2d.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, ci, cf, cf, ci, vp]
     lib.cg_diag_matmul.argtypes = [vp, vp, vp, vp, ctypes.c_longlong, ci, ci, vp]
     lib.cg_set_tuning.argtypes = [vp, ctypes.POINTER(cg_tuning_t)]
     lib.cg_set_trace.argtypes = [vp, vp, ci]
@@ -158,10 +158,12 @@ def cg_gemm_epilogue_ex(h, A, B, bias, R, D, M, N, K, batch, alpha, beta, act, r
                                       _stream_ptr(stream))
 
 
-def cg_conv2d(h, x, w, bias, R, y, n_img, H, W, IC, OC, KH, KW, pad_h=0, pad_w=0, alpha=1.0, beta=0.0, act=CG_ACT_NONE, stream=None) -> int:
-    """Stride-1 NHWC convolution as an implicit GEMM with the fused epilogue: x [n,H,W,IC], w [OC,KH,KW,IC], y [n,OH,OW,OC] (bf16)."""
+def cg_conv2d(h, x, w, bias, R, y, n_img, H, W, IC, OC, KH, KW, pad_h=0, pad_w=0, alpha=1.0, beta=0.0, act=CG_ACT_NONE, stream=None,
+              stride=1, dilation=1) -> int:
+    """NHWC convolution as an implicit GEMM with the fused epilogue: x [n,H,W,IC], w [OC,KH,KW,IC], y [n,OH,OW,OC] (bf16)."""
     return load().cg_conv2d(h, _dev_ptr(x), _dev_ptr(w), _dev_ptr(bias), _dev_ptr(R), _dev_ptr(y), int(n_img), int(H), int(W), int(IC),
-                            int(OC), int(KH), int(KW), int(pad_h), int(pad_w), float(alpha), float(beta), int(act), _stream_ptr(stream))
+                            int(OC), int(KH), int(KW), int(pad_h), int(pad_w), int(stride), int(dilation), float(alpha), float(beta), int(act),
+                            _stream_ptr(stream))
 
 
 def cg_diag_matmul(h, d, B, C, M, N, dtype=CG_OUT_BF16, stream=None) -> int:
@@ -233,8 +235,9 @@ class Context:
         if rc != CG_OK:
             raise CgError(rc, cg_last_error(self.handle)[1])
 
-    def conv2d(self, x, w, bias, R, y, n_img, H, W, IC, OC, KH, KW, pad_h=0, pad_w=0, alpha=1.0, beta=0.0, act=CG_ACT_NONE, stream=None):
-        rc = cg_conv2d(self.handle, x, w, bias, R, y, n_img, H, W, IC, OC, KH, KW, pad_h, pad_w, alpha, beta, act, stream)
+    def conv2d(self, x, w, bias, R, y, n_img, H, W, IC, OC, KH, KW, pad_h=0, pad_w=0, alpha=1.0, beta=0.0, act=CG_ACT_NONE, stream=None,
+               stride=1, dilation=1):
+        rc = cg_conv2d(self.handle, x, w, bias, R, y, n_img, H, W, IC, OC, KH, KW, pad_h, pad_w, alpha, beta, act, stream, stride, dilation)
         if rc != CG_OK:
             raise CgError(rc, cg_last_error(self.handle)[1])
 

@@ -227,12 +227,13 @@ int make_map(cg_context* h, CUtensorMap* map, const void* base, uint64_t inner, 
 }
 
 // bf16, rank 4 (channels, width, height, images), dense NHWC, 128-byte swizzle, zero fill outside the tensor.
+// `step` > 1: the box takes every step-th pixel in both directions (box_w x box_h pixels all the same).
 int make_map4(cg_context* h, CUtensorMap* map, const void* base, uint64_t c, uint64_t w, uint64_t hh, uint64_t n,
-              uint32_t box_c, uint32_t box_w, uint32_t box_h) {
+              uint32_t box_c, uint32_t box_w, uint32_t box_h, uint32_t step = 1) {
   const cuuint64_t dims[4] = {c, w, hh, n};
   const cuuint64_t strides[3] = {c * 2, c * w * 2, c * w * hh * 2};
-  const cuuint32_t box[4] = {box_c, box_w, box_h, 1};
-  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  const cuuint32_t box[4] = {box_c, box_w * step, box_h * step, 1};      // the box spans step x as many pixels as it loads
+  const cuuint32_t estr[4] = {1, step, step, 1};
   const CUresult r = h->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -490,7 +491,7 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   lookup(pl.bn, pl.cg, b_kmajor, &e, conv != nullptr);
 
   CUtensorMap tmA, tmB, tmD, tmR;
-  if (conv) rc = make_map4(h, &tmA, A, conv->IC, conv->W, conv->H, conv->n_img, BK, CONV_TILE_W, CONV_TILE_H);
+  if (conv) rc = make_map4(h, &tmA, A, conv->IC, conv->W, conv->H, conv->n_img, BK, CONV_TILE_W, CONV_TILE_H, conv->stride);
   else rc = make_map(h, &tmA, A, K, M, batch, bk_elems, BM, in_dtype);
   if (rc != CG_OK) return rc;
   const int b_entries = b_broadcast ? 1 : batch;
@@ -701,14 +702,17 @@ int cg_gemm_epilogue_ex(cg_handle_t h, const void* A, const void* B, const void*
 }
 
 int cg_conv2d(cg_handle_t h, const void* x, const void* w, const void* bias, const void* R, void* y, int n_img, int H, int W,
-              int IC, int OC, int KH, int KW, int pad_h, int pad_w, float alpha, float beta, int act, void* stream) {
+              int IC, int OC, int KH, int KW, int pad_h, int pad_w, int stride, int dilation, float alpha, float beta, int act,
+              void* stream) {
   if (!h) return CG_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lock(h->mu);
   if (!x || !w || !y) return fail(h, CG_ERR_INVALID_ARG, "x, w and y must not be NULL");
-  if (n_img < 1 || H < 1 || W < 1 || IC < 1 || OC < 1 || KH < 1 || KW < 1 || pad_h < 0 || pad_w < 0)
-    return fail(h, CG_ERR_INVALID_ARG, "sizes must be >= 1 and paddings >= 0");
-  const int OH = H + 2 * pad_h - KH + 1, OW = W + 2 * pad_w - KW + 1;
-  if (OH < 1 || OW < 1) return fail(h, CG_ERR_INVALID_ARG, "the filter does not fit the padded image");
+  if (n_img < 1 || H < 1 || W < 1 || IC < 1 || OC < 1 || KH < 1 || KW < 1 || pad_h < 0 || pad_w < 0 || stride < 1 || dilation < 1)
+    return fail(h, CG_ERR_INVALID_ARG, "sizes, stride and dilation must be >= 1 and paddings >= 0");
+  if (stride > 8) return fail(h, CG_ERR_UNSUPPORTED, "stride %d: the TMA box (16 * stride pixels wide) would exceed 256", stride);
+  const int span_h = (KH - 1) * dilation + 1, span_w = (KW - 1) * dilation + 1;       // extent of the dilated filter
+  if (H + 2 * pad_h < span_h || W + 2 * pad_w < span_w) return fail(h, CG_ERR_INVALID_ARG, "the filter does not fit the padded image");
+  const int OH = (H + 2 * pad_h - span_h) / stride + 1, OW = (W + 2 * pad_w - span_w) / stride + 1;
   const int kind = act & 0xFF;
   if (kind > CG_ACT_LEAKY_RELU || (act & ~(0xFF | CG_FLAG_BIAS_BF16)) != 0 || act < 0)
     return fail(h, CG_ERR_INVALID_ARG, "unknown activation or flag bits in act=0x%x", act);
@@ -719,6 +723,7 @@ int cg_conv2d(cg_handle_t h, const void* x, const void* w, const void* bias, con
   ConvGeom g;
   memset(&g, 0, sizeof g);
   g.on = 1; g.n_img = n_img; g.H = H; g.W = W; g.OH = OH; g.OW = OW; g.KH = KH; g.KW = KW; g.pad_h = pad_h; g.pad_w = pad_w; g.IC = IC;
+  g.stride = stride; g.dilation = dilation;
   g.ic_blocks = ceil_div(IC, BK);
   g.tiles_h = ceil_div(OH, CONV_TILE_H);
   g.tiles_w = ceil_div(OW, CONV_TILE_W);

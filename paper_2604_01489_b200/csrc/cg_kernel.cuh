@@ -76,11 +76,13 @@ enum { STATUS_OK = 0, STATUS_SMEM = 4, STATUS_TIMEOUT = 6 };
 
 // Implicit-GEMM convolution (stride 1, NHWC): output pixels are the GEMM's rows, in tiles of 8 x 16
 // pixels (128 rows); output channels its columns; K runs over (kh, kw, 64-channel block).  A k-block of
-// the A operand is one rank-4 TMA box of the input -- 64 channels x 16 x 8 pixels, shifted by the tap
-// and the padding; whatever falls outside the image is zero-filled by the TMA unit, which is the padding.
+// the A operand is one rank-4 TMA box of the input -- 64 channels x 16 x 8 pixels (every stride-th pixel:
+// the box's traversal stride), its origin shifted by the tap (times the dilation) and the padding; whatever
+// falls outside the image is zero-filled by the TMA unit, which is the padding.
 struct ConvGeom {
   int on;
   int n_img, H, W, OH, OW, KH, KW, pad_h, pad_w, IC;
+  int stride, dilation;   // same in both directions; the stride is the TMA box's traversal stride
   int ic_blocks;          // ceil(IC / 64)
   int tiles_h, tiles_w;   // pixel tiles per image
 };
@@ -441,7 +443,8 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       const int kh = tap / p.cv.KW, kw = tap - kh * p.cv.KW;
       int n, h0, w0;
       conv_strip(p, m0, n, h0, w0);
-      if (!withhold_a) ptx::tma_load_4d(a_dst, &tmA, bar, icb * BK, w0 - p.cv.pad_w + kw, h0 - p.cv.pad_h + kh, n);
+      if (!withhold_a) ptx::tma_load_4d(a_dst, &tmA, bar, icb * BK, w0 * p.cv.stride - p.cv.pad_w + kw * p.cv.dilation,
+                                        h0 * p.cv.stride - p.cv.pad_h + kh * p.cv.dilation, n);
       k0 = tap * p.cv.IC + icb * BK;                   // the weights' K index of this block
     } else if (!withhold_a) {
       ptx::tma_load_3d(a_dst, &tmA, bar, k0, m0, b);   // (withheld only by the starvation test hook)
@@ -528,7 +531,8 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
               const int kh = tap / p.cv.KW, kw = tap - kh * p.cv.KW;
               int n, h0, w0;
               conv_strip(p, m0, n, h0, w0);
-              ptx::tma_load_4d_pair(a_dst, &tmA, bar, icb * BK, w0 - p.cv.pad_w + kw, h0 - p.cv.pad_h + kh, n);
+              ptx::tma_load_4d_pair(a_dst, &tmA, bar, icb * BK, w0 * p.cv.stride - p.cv.pad_w + kw * p.cv.dilation,
+                                    h0 * p.cv.stride - p.cv.pad_h + kh * p.cv.dilation, n);
               k0 = tap * p.cv.IC + icb * BK;
             } else if (!(p.test_starve && issued == 0)) {
               ptx::tma_load_3d_pair(a_dst, &tmA, bar, k0, m0, b);

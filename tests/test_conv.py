@@ -12,11 +12,16 @@ def f64(b):
     return gen.bf16_bits_to_f32(b).astype(np.float64)
 
 
-def problem(n, H, Wd, IC, OC, KH, KW, seed, dist=("normal", 1.0), wdist=("normal", 0.2), bias=True, residual=False, ph=0, pw=0):
+def out_size(H, Wd, KH, KW, ph, pw, stride=1, dilation=1):
+    return (H + 2 * ph - (KH - 1) * dilation - 1) // stride + 1, (Wd + 2 * pw - (KW - 1) * dilation - 1) // stride + 1
+
+
+def problem(n, H, Wd, IC, OC, KH, KW, seed, dist=("normal", 1.0), wdist=("normal", 0.2), bias=True, residual=False, ph=0, pw=0,
+            stride=1, dilation=1):
     x = gen.tensor(seed, gen.TENSOR_A, (n, H, Wd, IC), dist[0], dist[1])
     w = gen.tensor(seed, gen.TENSOR_B, (OC, KH, KW, IC), wdist[0], wdist[1])
     b = gen.tensor(seed, gen.TENSOR_BIAS, (OC,), dist[0], dist[1], dtype="f32") if bias else None
-    OH, OW = H + 2 * ph - KH + 1, Wd + 2 * pw - KW + 1
+    OH, OW = out_size(H, Wd, KH, KW, ph, pw, stride, dilation)
     r = gen.tensor(seed, gen.TENSOR_R, (n, OH, OW, OC), dist[0], dist[1]) if residual else None
     return x, w, b, r
 
@@ -38,6 +43,24 @@ def test_oracle_conv_against_torch_fp64(oracle, geom):
     s64, _ = oracle.conv2d(x, w, b, None, ph, pw, alpha=0.75, act=W.ACT_SILU)
     t = 0.75 * torch.nn.functional.conv2d(xt, wt, None, padding=(ph, pw)) + torch.from_numpy(b.astype(np.float64))[None, :, None, None]
     assert np.allclose(s64, torch.nn.functional.silu(t).permute(0, 2, 3, 1).numpy(), rtol=1e-12, atol=1e-12)
+
+
+@pytest.mark.parametrize("sd", [(2, 1), (3, 1), (1, 2), (2, 2), (1, 3)], ids=lambda t: f"stride{t[0]}dil{t[1]}")
+def test_oracle_conv_stride_and_dilation_against_torch_fp64(oracle, sd):
+    import torch
+    stride, dilation = sd
+    n, H, Wd, IC, OC, KH, KW, ph, pw = 2, 13, 17, 8, 16, 3, 2, 2, 1
+    x, w, b, r = problem(n, H, Wd, IC, OC, KH, KW, seed=stride * 10 + dilation, residual=True, ph=ph, pw=pw, stride=stride, dilation=dilation)
+    y64, _ = oracle.conv2d(x, w, b, r, ph, pw, alpha=1.5, beta=0.25, act=W.ACT_NONE, stride=stride, dilation=dilation)
+    xt = torch.from_numpy(f64(x)).permute(0, 3, 1, 2)
+    wt = torch.from_numpy(f64(w)).permute(0, 3, 1, 2)
+    ref = 1.5 * torch.nn.functional.conv2d(xt, wt, None, stride=stride, padding=(ph, pw), dilation=dilation)
+    ref = (ref + torch.from_numpy(b.astype(np.float64))[None, :, None, None]).permute(0, 2, 3, 1).numpy() + 0.25 * f64(r)
+    assert y64.shape == ref.shape and np.allclose(y64, ref, rtol=1e-12, atol=1e-12)
+    # a stride-s convolution is the stride-1 one sampled at every s-th output pixel
+    full64, _ = oracle.conv2d(x, w, b, None, ph, pw, alpha=1.5, act=W.ACT_NONE, stride=1, dilation=dilation)
+    sub64, _ = oracle.conv2d(x, w, b, None, ph, pw, alpha=1.5, act=W.ACT_NONE, stride=stride, dilation=dilation)
+    assert np.array_equal(sub64, full64[:, ::stride, ::stride][:, :sub64.shape[1], :sub64.shape[2]])
 
 
 def test_oracle_conv_special_cases(oracle):
@@ -85,15 +108,15 @@ def ctx():
     c.close()
 
 
-def run_conv(ctx, x, w, b, r, ph, pw, alpha, beta, act):
+def run_conv(ctx, x, w, b, r, ph, pw, alpha, beta, act, stride=1, dilation=1):
     import torch
     to = lambda a: None if a is None else torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
     n, H, Wd, IC = x.shape
     OC, KH, KW, _ = w.shape
-    OH, OW = H + 2 * ph - KH + 1, Wd + 2 * pw - KW + 1
+    OH, OW = out_size(H, Wd, KH, KW, ph, pw, stride, dilation)
     y = torch.full((n, OH, OW, OC), float("nan"), dtype=torch.bfloat16, device="cuda")
     bd = None if b is None else torch.from_numpy(b).cuda()
-    ctx.conv2d(to(x), to(w), bd, to(r), y, n, H, Wd, IC, OC, KH, KW, ph, pw, alpha, beta, act)
+    ctx.conv2d(to(x), to(w), bd, to(r), y, n, H, Wd, IC, OC, KH, KW, ph, pw, alpha, beta, act, stride=stride, dilation=dilation)
     ctx.check()
     return y.view(torch.int16).cpu().numpy().view(np.uint16)
 
@@ -119,6 +142,23 @@ def test_gpu_conv_integer_operands_bit_exact(ctx, oracle, geom, plan):
     assert np.array_equal(y, y16), int(np.sum(y != y16))
     pl = ctx.last_plan()
     assert pl["k_blocks"] == KH * KW * ((IC + 63) // 64) and pl["latency_kernel"] == 0
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("plan", [dict(), dict(tile_n=256, cta_group=2), dict(tile_n=128, cta_group=1, num_units=11)],
+                         ids=lambda d: "auto" if not d else "-".join(f"{k}{v}" for k, v in d.items()))
+@pytest.mark.parametrize("sd", [(2, 1), (3, 1), (1, 2), (2, 2), (4, 3)], ids=lambda t: f"stride{t[0]}dil{t[1]}")
+def test_gpu_conv_stride_and_dilation_bit_exact(ctx, oracle, sd, plan):
+    stride, dilation = sd
+    n, H, Wd, IC, OC, KH, KW, ph, pw = 2, 41, 67, 72, 136, 3, 3, 2, 1
+    x, w, b, r = problem(n, H, Wd, IC, OC, KH, KW, seed=stride * 7 + dilation, dist=(SI, 1.0), wdist=(SI, 1.0), residual=True, ph=ph, pw=pw,
+                         stride=stride, dilation=dilation)
+    ctx.set_tuning(reset=True)
+    if plan:
+        ctx.set_tuning(**plan)
+    y = run_conv(ctx, x, w, b, r, ph, pw, 2.0, -1.0, W.ACT_RELU, stride=stride, dilation=dilation)
+    _, y16 = oracle.conv2d(x, w, b, r, ph, pw, alpha=2.0, beta=-1.0, act=W.ACT_RELU, stride=stride, dilation=dilation)
+    assert y.shape == y16.shape and np.array_equal(y, y16), int(np.sum(y != y16))
 
 
 @pytest.mark.gpu
@@ -150,5 +190,8 @@ def test_gpu_conv_error_codes(ctx):
     assert cg.cg_conv2d(h, x, w, None, None, y, 1, 8, 8, 8, 8, 3, 3, beta=1.0) == cg.CG_ERR_INVALID_ARG
     assert cg.cg_conv2d(h, x, w, None, None, y, 1, 8, 8, 4, 8, 3, 3) == cg.CG_ERR_UNSUPPORTED       # IC % 8
     assert cg.cg_conv2d(h, x, w, None, None, y, 1, 8, 8, 8, 8, 3, 3, act=cg.CG_FLAG_B_COLMAJOR) == cg.CG_ERR_INVALID_ARG
+    assert cg.cg_conv2d(h, x, w, None, None, y, 1, 8, 8, 8, 8, 3, 3, stride=0) == cg.CG_ERR_INVALID_ARG
+    assert cg.cg_conv2d(h, x, w, None, None, y, 1, 8, 8, 8, 8, 3, 3, dilation=4) == cg.CG_ERR_INVALID_ARG  # dilated filter larger than the image
+    assert cg.cg_conv2d(h, x, w, None, None, y, 1, 8, 8, 8, 8, 3, 3, stride=9) == cg.CG_ERR_UNSUPPORTED
     assert cg.cg_conv2d(h, x, w, None, None, y, 1, 8, 8, 8, 8, 3, 3) == cg.CG_OK
     ctx.check()
