@@ -162,6 +162,24 @@ def test_gpu_conv_stride_and_dilation_bit_exact(ctx, oracle, sd, plan):
 
 
 @pytest.mark.gpu
+@pytest.mark.parametrize("geom", [(1, 8, 8, 8, 8, 3, 3, 1, 1), (1, 3, 5, 16, 24, 3, 3, 1, 1), (3, 1, 1, 64, 64, 1, 1, 0, 0), (1, 4, 40, 8, 520, 1, 7, 0, 3),
+                                  (5, 7, 9, 200, 72, 2, 2, 0, 0)], ids=str)
+def test_gpu_conv_small_and_odd_geometries(ctx, oracle, geom):
+    """Images smaller than a pixel tile, a single pixel, an odd number of pixel tiles under CTA pairs, wide flat filters."""
+    n, H, Wd, IC, OC, KH, KW, ph, pw = geom
+    x, w, b, r = problem(n, H, Wd, IC, OC, KH, KW, seed=sum(geom), dist=(SI, 1.0), wdist=(SI, 1.0), residual=True, ph=ph, pw=pw)
+    _, y16 = oracle.conv2d(x, w, b, r, ph, pw, alpha=1.0, beta=1.0, act=W.ACT_LEAKY_RELU)
+    for plan in (dict(), dict(tile_n=128, cta_group=2), dict(tile_n=64, cta_group=1)):
+        ctx.set_tuning(reset=True)
+        if plan:
+            ctx.set_tuning(**plan)
+        y = run_conv(ctx, x, w, b, r, ph, pw, 1.0, 1.0, W.ACT_LEAKY_RELU)
+        # leaky ReLU's slope 0.01 is not a power of two: the negative side is rounded once more on the GPU (fp32, then bf16)
+        diff = np.abs(y.astype(np.int32) - y16.astype(np.int32))
+        assert diff.max() <= 1, (plan, int(diff.max()))
+
+
+@pytest.mark.gpu
 @pytest.mark.parametrize("act", [W.ACT_NONE, W.ACT_GELU_TANH, W.ACT_SILU])
 def test_gpu_conv_random_inputs(ctx, oracle, act):
     import parity_util as PU
