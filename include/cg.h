@@ -180,6 +180,10 @@ CG_API int cg_diag_matmul(cg_handle_t h, const float* d, const void* B, void* C,
  * pinned memory makes the copies asynchronous and faster).  Copies the operands to device
  * staging buffers owned by the handle (grown on demand and kept), runs the kernel, copies D
  * back and synchronises `stream` before returning.  The end-to-end path of the benchmark.
+ * Problems with batch >= 2 or M >= 2048 travel in up to eight chunks (batch entries, or row blocks of
+ * 256 rows): chunk i+1 is copied in on one internal stream while chunk i is computed on `stream` and
+ * chunk i-1 is copied out on another, so the call costs about the larger of the two copy directions
+ * instead of their sum plus the kernel.
  */
 CG_API int cg_gemm_epilogue_host(cg_handle_t h, const void* A, const void* B, const void* bias, const void* R,
                           void* D, int M, int N, int K, int batch, float alpha, float beta, int act,

@@ -97,6 +97,11 @@ struct cg_context {
   int map_cache_next = 0;
   StagingBuf sA, sB, sBias, sR, sD;
   StagingBuf row_ws;                     // partial results of fused row reductions
+  // the host-buffer entry point overlaps its copies with the kernels: copy streams and events, made on first use
+  static constexpr int HOST_CHUNKS = 8;
+  cudaStream_t s_h2d = nullptr, s_d2h = nullptr;
+  cudaEvent_t ev_start = nullptr, ev_shared = nullptr, ev_done = nullptr, ev_in[HOST_CHUNKS] = {}, ev_out[HOST_CHUNKS] = {};
+  int host_pipeline = 1;                 // CG_HOST_PIPELINE=0: one copy-in, one launch, one copy-out (ablation)
   std::mutex mu;
 };
 
@@ -465,6 +470,8 @@ int launch_small(cg_context* h, const void* A, const void* B, const void* bias, 
 }
 
 int grow(cg_context* h, StagingBuf* s, size_t bytes);
+int host_pipelined(cg_context* h, const char* A, const char* B, const void* bias, const char* R, char* D, int M, int N, int K,
+                   int batch, float alpha, float beta, int act, cudaStream_t st);
 
 int launch(cg_context* h, const void* A, const void* B, const void* bias, const void* R, void* D, int M, int N, int K,
            int batch, float alpha, float beta, int act, cudaStream_t stream, const cg_epilogue_ex_t* ex = nullptr,
@@ -609,6 +616,73 @@ int grow(cg_context* h, StagingBuf* s, size_t bytes) {
   return CG_OK;
 }
 
+// The same with the problem cut into up to eight chunks -- batch entries, or row blocks of a single GEMM -- so
+// that chunk i+1 travels to the device while chunk i is computed and chunk i-1 travels back (PCIe is full
+// duplex and the copies, not the kernel, are what the call costs).  Three streams: copies in, the caller's
+// stream for the kernels, copies out; events order them.  Returns -1 when the problem is not worth cutting.
+int host_pipelined(cg_context* h, const char* A, const char* B, const void* bias, const char* R, char* D, int M, int N, int K,
+                   int batch, float alpha, float beta, int act, cudaStream_t st) {
+  constexpr int MAXC = cg_context::HOST_CHUNKS;
+  const bool by_batch = batch >= 2;
+  if (!h->host_pipeline || (!by_batch && M < 2048)) return -1;
+  if (!h->s_h2d) {
+    CG_CUDA(h, cudaStreamCreateWithFlags(&h->s_h2d, cudaStreamNonBlocking));
+    CG_CUDA(h, cudaStreamCreateWithFlags(&h->s_d2h, cudaStreamNonBlocking));
+    cudaEvent_t* evs[3] = {&h->ev_start, &h->ev_shared, &h->ev_done};
+    for (cudaEvent_t* e : evs) CG_CUDA(h, cudaEventCreateWithFlags(e, cudaEventDisableTiming));
+    for (int i = 0; i < MAXC; ++i) {
+      CG_CUDA(h, cudaEventCreateWithFlags(&h->ev_in[i], cudaEventDisableTiming));
+      CG_CUDA(h, cudaEventCreateWithFlags(&h->ev_out[i], cudaEventDisableTiming));
+    }
+  }
+  // chunk c covers units [c * per, min((c + 1) * per, total)): batch entries, or rows in multiples of 256
+  const int total = by_batch ? batch : M;
+  int per = (total + MAXC - 1) / MAXC;
+  if (!by_batch) per = (per + 255) / 256 * 256;
+  const int chunks = (total + per - 1) / per;
+  const size_t row_a = static_cast<size_t>(K) * 2, row_d = static_cast<size_t>(N) * 2;
+  const size_t unit_a = by_batch ? static_cast<size_t>(M) * row_a : row_a, unit_d = by_batch ? static_cast<size_t>(M) * row_d : row_d;
+  const size_t unit_b = static_cast<size_t>(K) * N * 2;            // one batch entry of B
+  const size_t bias_bytes = bias ? static_cast<size_t>(N) * ((act & CG_FLAG_BIAS_BF16) ? 2 : 4) : 0;
+  const bool use_r = beta != 0.0f;
+  char* dA = static_cast<char*>(h->sA.ptr);
+  char* dB = static_cast<char*>(h->sB.ptr);
+  char* dR = static_cast<char*>(h->sR.ptr);
+  char* dD = static_cast<char*>(h->sD.ptr);
+
+  CG_CUDA(h, cudaEventRecord(h->ev_start, st));                      // everything here follows the caller's earlier work
+  CG_CUDA(h, cudaStreamWaitEvent(h->s_h2d, h->ev_start, 0));
+  CG_CUDA(h, cudaStreamWaitEvent(h->s_d2h, h->ev_start, 0));
+  if (bias) CG_CUDA(h, cudaMemcpyAsync(h->sBias.ptr, bias, bias_bytes, cudaMemcpyHostToDevice, h->s_h2d));
+  if (!by_batch) CG_CUDA(h, cudaMemcpyAsync(dB, B, unit_b, cudaMemcpyHostToDevice, h->s_h2d));     // B is shared by the row blocks
+  CG_CUDA(h, cudaEventRecord(h->ev_shared, h->s_h2d));
+  CG_CUDA(h, cudaStreamWaitEvent(st, h->ev_shared, 0));
+  for (int c = 0; c < chunks; ++c) {
+    const int u0 = c * per, n = (u0 + per <= total ? per : total - u0);
+    CG_CUDA(h, cudaMemcpyAsync(dA + u0 * unit_a, A + u0 * unit_a, n * unit_a, cudaMemcpyHostToDevice, h->s_h2d));
+    if (by_batch) CG_CUDA(h, cudaMemcpyAsync(dB + u0 * unit_b, B + u0 * unit_b, n * unit_b, cudaMemcpyHostToDevice, h->s_h2d));
+    if (use_r) CG_CUDA(h, cudaMemcpyAsync(dR + u0 * unit_d, R + u0 * unit_d, n * unit_d, cudaMemcpyHostToDevice, h->s_h2d));
+    CG_CUDA(h, cudaEventRecord(h->ev_in[c], h->s_h2d));
+    CG_CUDA(h, cudaStreamWaitEvent(st, h->ev_in[c], 0));
+    const int rc = launch(h, dA + u0 * unit_a, by_batch ? dB + u0 * unit_b : dB, bias ? h->sBias.ptr : nullptr,
+                          use_r ? dR + u0 * unit_d : nullptr, dD + u0 * unit_d, by_batch ? M : n, N, K, by_batch ? n : 1, alpha, beta,
+                          act, st);
+    if (rc != CG_OK) {
+      cudaStreamSynchronize(h->s_h2d);
+      cudaStreamSynchronize(h->s_d2h);
+      cudaStreamSynchronize(st);
+      return rc;
+    }
+    CG_CUDA(h, cudaEventRecord(h->ev_out[c], st));
+    CG_CUDA(h, cudaStreamWaitEvent(h->s_d2h, h->ev_out[c], 0));
+    CG_CUDA(h, cudaMemcpyAsync(D + u0 * unit_d, dD + u0 * unit_d, n * unit_d, cudaMemcpyDeviceToHost, h->s_d2h));
+  }
+  CG_CUDA(h, cudaEventRecord(h->ev_done, h->s_d2h));
+  CG_CUDA(h, cudaStreamWaitEvent(st, h->ev_done, 0));
+  CG_CUDA(h, cudaStreamSynchronize(st));
+  return CG_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -660,6 +734,7 @@ int cg_create(cg_handle_t* out, int device, size_t workspace_bytes) {
   if (const char* w = getenv("CG_SPLIT_FIRST")) h->split_first = atoi(w);
   if (const char* w = getenv("CG_WARM_UP")) h->warm_up = atoi(w);
   if (const char* w = getenv("CG_SMALL")) h->small_kernel = atoi(w);
+  if (const char* w = getenv("CG_HOST_PIPELINE")) h->host_pipeline = atoi(w);
   *out = h;
   return CG_OK;
 }
@@ -777,6 +852,9 @@ int cg_gemm_epilogue_host(cg_handle_t h, const void* A, const void* B, const voi
       (rc = grow(h, &h->sD, d_bytes)) != CG_OK || (bias && (rc = grow(h, &h->sBias, bias_bytes)) != CG_OK) ||
       (use_r && (rc = grow(h, &h->sR, d_bytes)) != CG_OK))
     return rc;
+  rc = host_pipelined(h, static_cast<const char*>(A), static_cast<const char*>(B), bias, static_cast<const char*>(R),
+                      static_cast<char*>(D), M, N, K, batch, alpha, beta, act, st);
+  if (rc >= 0) return rc;
   CG_CUDA(h, cudaMemcpyAsync(h->sA.ptr, A, a_bytes, cudaMemcpyHostToDevice, st));
   CG_CUDA(h, cudaMemcpyAsync(h->sB.ptr, B, b_bytes, cudaMemcpyHostToDevice, st));
   if (bias) CG_CUDA(h, cudaMemcpyAsync(h->sBias.ptr, bias, bias_bytes, cudaMemcpyHostToDevice, st));
@@ -851,6 +929,12 @@ int cg_destroy(cg_handle_t h) {
   cudaSetDevice(h->device);
   cudaFree(h->workspace);
   cudaFree(h->status);
+  if (h->s_h2d) {
+    cudaStreamDestroy(h->s_h2d);
+    cudaStreamDestroy(h->s_d2h);
+    cudaEventDestroy(h->ev_start); cudaEventDestroy(h->ev_shared); cudaEventDestroy(h->ev_done);
+    for (int i = 0; i < cg_context::HOST_CHUNKS; ++i) { cudaEventDestroy(h->ev_in[i]); cudaEventDestroy(h->ev_out[i]); }
+  }
   StagingBuf* bufs[6] = {&h->sA, &h->sB, &h->sBias, &h->sR, &h->sD, &h->row_ws};
   for (StagingBuf* s : bufs)
     if (s->ptr) cudaFree(s->ptr);

@@ -151,6 +151,31 @@ def test_host_buffer_entry_point(cg, ctx, oracle):
     assert PU.compare(d, r64)["ok"]
 
 
+@pytest.mark.parametrize("shape", [(2300, 264, 136, 1), (130, 72, 264, 11), (4096, 512, 64, 1)], ids=lambda t: "x".join(map(str, t)))
+def test_host_buffer_entry_point_pipelined_chunks(cg, ctx, oracle, shape):
+    """Large problems travel in up to eight chunks (row blocks or batch entries) that overlap with the kernels: ragged
+    last chunks, residual, pinned and pageable buffers; against the oracle and the device-buffer call."""
+    import torch
+    M, N, K, batch = shape
+    p = W.make(M, N, K, batch, seed=M + batch, act=W.ACT_SILU, alpha=0.5, beta=1.0, A=("normal", 1.0), B=("normal", 0.1),
+               bias=("normal", 1.0), R=("normal", 1.0))
+    ctx.set_tuning(reset=True)
+    want = PU.run_gpu(ctx, p)                                            # device buffers, one launch
+    d = np.zeros((batch, M, N), dtype=np.uint16)
+    ctx.gemm_epilogue_host(p.A, p.B, p.bias, p.R, d, M, N, K, batch, p.alpha, p.beta, p.act)
+    rows = W.sample_rows(p, 64)
+    r64, _ = PU.oracle_rows(oracle, p, rows)
+    assert PU.compare(d.reshape(-1, N)[rows], r64)["ok"]
+    # (a chunk may run under another plan, or the latency kernel, than the whole problem does: the last bit may differ)
+    diff = np.abs(d.astype(np.int32) - want.astype(np.int32))
+    assert diff.max() <= 1 and np.mean(diff != 0) < 0.01
+    pin = lambda a: torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a).pin_memory()
+    hd = torch.zeros((batch, M, N), dtype=torch.int16).pin_memory()
+    ctx.gemm_epilogue_host(pin(p.A), pin(p.B), pin(p.bias), pin(p.R), hd, M, N, K, batch, p.alpha, p.beta, p.act)
+    assert np.array_equal(hd.numpy().view(np.uint16), d)
+    ctx.check()
+
+
 STARVE_SCRIPT = r"""
 import os, sys
 sys.path.insert(0, {root!r}); sys.path.insert(0, os.path.join({root!r}, "tests"))
