@@ -154,7 +154,15 @@ struct Cfg {
   static constexpr int EPI_WARPS = (BN >= 128) ? 8 : 4;
   static constexpr int EPI_COL_GROUPS = EPI_WARPS / 4;       // warps per TMEM lane quarter
   static constexpr int EPI_BUFS = (EPI_WARPS == 4) ? 2 : 1;  // staging buffers per warp
-  static constexpr int NUM_THREADS = 64 + 32 * EPI_WARPS;
+  // The 512-wide tile's only accumulator is exposed while it drains, so its epilogue warps hold two
+  // chunks in registers (one being finished, one on its way out of tensor memory) and hand the
+  // accumulator back a chunk earlier.  The registers come from the producer / MMA warps: those
+  // form a warpgroup of their own (two of its warps idle) that gives up all but REGS_LEAD registers
+  // per thread, and the two epilogue warpgroups grow to REGS_EPI.
+  static constexpr bool DRAIN_AHEAD = (BN == 512);
+  static constexpr int LEAD_WARPS = DRAIN_AHEAD ? 4 : 2;       // warps before the first epilogue warp
+  static constexpr int REGS_LEAD = 40, REGS_EPI = 232;         // (128 * 40 + 256 * 232 = 384 * 168)
+  static constexpr int NUM_THREADS = 32 * (LEAD_WARPS + EPI_WARPS);
   static constexpr int EPI_BYTES = EPI_WARPS * EPI_BUFS * EPI_BUF_BYTES;
   static constexpr int BIAS_BYTES = EPI_WARPS * EPI_COLS * 4;   // per warp: one chunk of fp32 bias
   static constexpr int R_BYTES = EPI_WARPS * EPI_BUF_BYTES;      // per warp: one 64-column chunk of the residual
@@ -533,6 +541,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 
   if (warp == 0) {
     // ================================================================ producer
+    if constexpr (C::DRAIN_AHEAD) ptx::setmaxnreg_dec<C::REGS_LEAD>();   // (every warp of a warpgroup executes the same form)
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
@@ -616,6 +625,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     }
   } else if (warp == 1) {
     // ================================================================ MMA issuer
+    if constexpr (C::DRAIN_AHEAD) ptx::setmaxnreg_dec<C::REGS_LEAD>();
     // One thread feeds the tensor pipe, so its instruction count per k-block is what bounds
     // small tiles: descriptor words are precomputed and only their low (address) half moves.
     // (the role is instantiated twice, for bf16 and for TF32 operands: the choice of MMA instruction is
@@ -703,9 +713,10 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       ptx::cluster_arrive(); ptx::cluster_wait();
       ptx::cluster_arrive(); ptx::cluster_wait();
     }
-  } else {
-    // ================================================================ epilogue (warps 2 and up)
-    const int ew = warp - 2;                    // epilogue warp index
+  } else if (warp >= C::LEAD_WARPS) {
+    // ================================================================ epilogue (warps LEAD_WARPS and up)
+    if constexpr (C::DRAIN_AHEAD) ptx::setmaxnreg_inc<C::REGS_EPI>();
+    const int ew = warp - C::LEAD_WARPS;        // epilogue warp index
     const int q = warp & 3;                     // TMEM lane quarter this warp may access
     const int col_group = ew >> 2;              // which share of the tile's columns (wide tiles have two)
     const int row_in_tile = q * 32 + lane;
@@ -956,6 +967,24 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       }
 
       if (whole_tile || reduce || csk > 1) {
+        // hand-back of this warp's share of the accumulator to the MMA warp (after its last tcgen05.ld)
+        auto release_acc = [&]() {
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) {
+            if constexpr (CG == 2) ptx::mbar_arrive_cluster(acc_empty_bar); else ptx::mbar_arrive(acc_empty_bar);
+          }
+        };
+        // Drain ahead (512-wide tile): the chunk after the one being finished is already on its way
+        // from tensor memory into a second set of registers.
+        uint32_t nx0[32], nx1[32];
+        if constexpr (C::DRAIN_AHEAD) {
+          if (whole_tile && c_lo < c_hi) {
+            ptx::tmem_ld_32x32b_x32(taddr + c_lo * EPI_COLS, nx0);
+            ptx::tmem_ld_32x32b_x32(taddr + c_lo * EPI_COLS + 32, nx1);
+            if (c_lo + 1 == c_hi && !dry) { ptx::tmem_ld_wait(); release_acc(); }
+          }
+        }
         int c_ord = 0;             // position of the chunk in this warp's list
         for (int c = c_lo; c < c_hi; c += c_step, ++c_ord) {
           const int n0 = n_base + c * EPI_COLS;
@@ -975,18 +1004,28 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
               }
             }
           } else if (whole_tile) {
-            uint32_t v0[32], v1[32];
-            ptx::tmem_ld_32x32b_x32(taddr + c * EPI_COLS, v0);
-            ptx::tmem_ld_32x32b_x32(taddr + c * EPI_COLS + 32, v1);
-            ptx::tmem_ld_wait();
+            if constexpr (C::DRAIN_AHEAD) {
+              ptx::tmem_ld_wait();                 // the loads issued a chunk ago
 #pragma unroll
-            for (int j = 0; j < 32; ++j) { accv[j] = __uint_as_float(v0[j]); accv[32 + j] = __uint_as_float(v1[j]); }
-            if (c == c_hi - 1 && !dry) { // this warp's share is read: its hand-back of the buffer to the MMA warp
-              ptx::tc_fence_before();
-              __syncwarp();
-              if (lane == 0) {
-                if constexpr (CG == 2) ptx::mbar_arrive_cluster(acc_empty_bar); else ptx::mbar_arrive(acc_empty_bar);
+              for (int j = 0; j < 32; ++j) {
+                ptx::after_wait(nx0[j]);
+                ptx::after_wait(nx1[j]);
+                accv[j] = __uint_as_float(nx0[j]);
+                accv[32 + j] = __uint_as_float(nx1[j]);
               }
+              if (c + 1 < c_hi) {
+                ptx::tmem_ld_32x32b_x32(taddr + (c + 1) * EPI_COLS, nx0);
+                ptx::tmem_ld_32x32b_x32(taddr + (c + 1) * EPI_COLS + 32, nx1);
+                if (c + 2 == c_hi && !dry) { ptx::tmem_ld_wait(); release_acc(); }   // the last loads: waited for at once
+              }
+            } else {
+              uint32_t v0[32], v1[32];
+              ptx::tmem_ld_32x32b_x32(taddr + c * EPI_COLS, v0);
+              ptx::tmem_ld_32x32b_x32(taddr + c * EPI_COLS + 32, v1);
+              ptx::tmem_ld_wait();
+#pragma unroll
+              for (int j = 0; j < 32; ++j) { accv[j] = __uint_as_float(v0[j]); accv[32 + j] = __uint_as_float(v1[j]); }
+              if (c == c_hi - 1 && !dry) release_acc();   // this warp's share is read
             }
           } else {
 #pragma unroll
@@ -1131,6 +1170,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           store_buf = (store_buf + 1 == C::EPI_BUFS) ? 0 : store_buf + 1;
           if (r_shared && !dry) request_next_residual(c, c_step, c_hi, n0, m_base + q * 32, b, have_next, s_next, c_lo);
         }
+        if constexpr (C::DRAIN_AHEAD) ptx::tmem_ld_wait();   // (only when leaving the loop early)
         if (p.row_reduce && !dry && ok) {      // this row's partial over this warp's columns (identity if it had none)
           const int m = m_base + row_in_tile;
           if (m < p.M) {
@@ -1143,13 +1183,7 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             }
           }
         }
-        if (whole_tile && c_lo >= c_hi && !dry) {    // none of this warp's columns exist (ragged N): still hand the buffer back
-          ptx::tc_fence_before();
-          __syncwarp();
-          if (lane == 0) {
-            if constexpr (CG == 2) ptx::mbar_arrive_cluster(acc_empty_bar); else ptx::mbar_arrive(acc_empty_bar);
-          }
-        }
+        if (whole_tile && c_lo >= c_hi && !dry) release_acc();   // none of this warp's columns exist (ragged N)
       }
       if (dry) {
         dry = 0;
@@ -1171,6 +1205,8 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     if (lane == 0) ptx::bulk_wait_group_read<0>();
     if (ew == 0 && lane == 0) trace_event(p, TR_STORES_DONE);
     __syncwarp();
+  } else if constexpr (C::DRAIN_AHEAD) {
+    ptx::setmaxnreg_dec<C::REGS_LEAD>();        // the idle warps of the first warpgroup
   }
 
   // ---- tear-down

@@ -237,6 +237,13 @@ __device__ __forceinline__ void tmem_ld_32x32b_x16(uint32_t taddr, uint32_t (&v)
       : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// Ties a register that an earlier tcgen05.ld fills to the wait before it (no instruction): volatile
+// statements keep their order, so nothing that uses the value can move ahead of the wait.
+__device__ __forceinline__ void after_wait(uint32_t& v) { asm volatile("" : "+r"(v)::"memory"); }
+
+// Per-thread register budget of the executing warpgroup (all four warps run the same instruction).
+template <int N> __device__ __forceinline__ void setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void setmaxnreg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 
 __device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
