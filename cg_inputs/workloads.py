@@ -26,6 +26,7 @@ FLAG_BIAS_PER_ROW = 1 << 10
 FLAG_B_BROADCAST = 1 << 11
 FLAG_CLAMP = 1 << 12
 FLAG_IN_F32 = 1 << 13
+FLAG_A_SYMMETRIC = 1 << 14
 OUT_BF16, OUT_F16, OUT_F32 = 0, 1, 2
 
 
@@ -54,7 +55,7 @@ class Problem:
 
     @property
     def extended(self) -> bool:
-        return bool(self.act & (FLAG_BIAS_PER_ROW | FLAG_B_BROADCAST | FLAG_CLAMP | FLAG_IN_F32)) or self.row_scale is not None \
+        return bool(self.act & (FLAG_BIAS_PER_ROW | FLAG_B_BROADCAST | FLAG_CLAMP | FLAG_IN_F32 | FLAG_A_SYMMETRIC)) or self.row_scale is not None \
             or self.col_scale is not None or self.out_dtype != OUT_BF16
 
     @property
@@ -103,10 +104,16 @@ def make(M, N, K, batch=1, seed=0, act=ACT_NONE, alpha=1.0, beta=0.0, A=("unifor
          out_dtype=OUT_BF16) -> Problem:
     """Build a problem from distribution specs (see CONFIGS for the format).  ``row_scale`` /
     ``col_scale``: distribution specs of fp32 vectors ("pow2" draws exact powers of two 2^-2..2^2);
-    ``clamp``: (lo, hi), sets FLAG_CLAMP."""
+    ``clamp``: (lo, hi), sets FLAG_CLAMP.  With FLAG_A_SYMMETRIC A is made symmetric by mirroring its upper
+    triangle (see also ``poison_below_blocks``)."""
     colmajor = bool(act & FLAG_B_COLMAJOR)
     in_dtype = "f32" if act & FLAG_IN_F32 else "bf16"
     a = gen.tensor(seed, gen.TENSOR_A, (batch, M, K), A[0], A[1], dtype=in_dtype)
+    if act & FLAG_A_SYMMETRIC:
+        if M != K:
+            raise ValueError("a symmetric A is square")
+        iu = np.triu_indices(M, 1)
+        a[:, iu[1], iu[0]] = a[:, iu[0], iu[1]]
     b = gen.tensor(seed, gen.TENSOR_B, (1 if act & FLAG_B_BROADCAST else batch, K, N), B[0], B[1], dtype=in_dtype,
                    colmajor_last2=colmajor)
     bias_arr = None
@@ -135,6 +142,17 @@ def make(M, N, K, batch=1, seed=0, act=ACT_NONE, alpha=1.0, beta=0.0, A=("unifor
                    bias=bias_arr, R=r, seed=seed, row_scale=scale_vec(row_scale, gen.TENSOR_ROW_SCALE, M),
                    col_scale=scale_vec(col_scale, gen.TENSOR_COL_SCALE, N), clamp_lo=float(lo), clamp_hi=float(hi),
                    out_dtype=out_dtype)
+
+
+def poison_below_blocks(a: np.ndarray, block: int, bits: int = 0x7FC0) -> np.ndarray:
+    """Copy of the square matrices ``a`` [batch, M, M] (bf16 bits) in which every element below the diagonal and
+    outside the block x block squares on the diagonal is a NaN: what a kernel that honours the symmetric flag
+    at that block size never reads."""
+    out = a.copy()
+    m = a.shape[-1]
+    i, k = np.meshgrid(np.arange(m), np.arange(m), indexing="ij")
+    out[:, (i // block) > (k // block)] = bits
+    return out
 
 
 def config(name: str) -> Problem:

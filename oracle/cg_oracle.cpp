@@ -99,7 +99,7 @@ enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU_TANH = 2, ACT_SILU = 3,
 constexpr int ACT_LAST = ACT_LEAKY_RELU;
 constexpr double LEAKY_SLOPE = 0.01;
 enum { FLAG_B_COLMAJOR = 1 << 8, FLAG_BIAS_BF16 = 1 << 9, FLAG_BIAS_PER_ROW = 1 << 10, FLAG_B_BROADCAST = 1 << 11,
-       FLAG_CLAMP = 1 << 12, FLAG_IN_F32 = 1 << 13 };
+       FLAG_CLAMP = 1 << 12, FLAG_IN_F32 = 1 << 13, FLAG_A_SYMMETRIC = 1 << 14 };
 enum { OUT_BF16 = 0, OUT_F16 = 1, OUT_F32 = 2 };
 enum { REDUCE_NONE = 0, REDUCE_SUM = 1, REDUCE_MAX = 2, REDUCE_LOGSUMEXP = 3 };
 
@@ -168,7 +168,7 @@ struct Problem {
   int act;
   bool b_colmajor, bias_bf16;
   // extended family (all off in the base entry points)
-  bool bias_per_row = false, b_broadcast = false, clamp = false, in_f32 = false;
+  bool bias_per_row = false, b_broadcast = false, clamp = false, in_f32 = false, a_symmetric = false;
   const float* row_scale = nullptr;   // [M] or null
   const float* col_scale = nullptr;   // [N] or null
   double clamp_lo = 0.0, clamp_hi = 0.0;
@@ -188,7 +188,13 @@ inline double operand(const Problem& p, const void* base, int64_t i) {
   if (p.in_f32) return f32_as_tf32(static_cast<const float*>(base)[i]);
   return bf16_to_f64(static_cast<const uint16_t*>(base)[i]);
 }
-inline double a_at(const Problem& p, int64_t b, int64_t m, int64_t k) { return operand(p, p.A, (b * p.M + m) * p.K + k); }
+// A[b,m,k].  Under the symmetric flag (square A; the GEMM prompt's hint that a symmetric operand needs fewer
+// reads) the upper triangle is the matrix: an element below the diagonal is its mirror image above it, and what
+// the array holds there is never looked at.
+inline double a_at(const Problem& p, int64_t b, int64_t m, int64_t k) {
+  if (p.a_symmetric && m > k) return operand(p, p.A, (b * p.M + k) * p.K + m);
+  return operand(p, p.A, (b * p.M + m) * p.K + k);
+}
 
 // B[b,k,n] through an index function: row-major [batch,K,N] or column-major [batch,N,K];
 // a shared B has a single batch entry.
@@ -271,6 +277,7 @@ Problem make_ex(const void* A, const void* B, const void* bias, const void* R, i
   p.b_broadcast = (act & FLAG_B_BROADCAST) != 0;
   p.clamp = (act & FLAG_CLAMP) != 0;
   p.in_f32 = (act & FLAG_IN_F32) != 0;
+  p.a_symmetric = (act & FLAG_A_SYMMETRIC) != 0;
   p.row_scale = row_scale;
   p.col_scale = col_scale;
   p.clamp_lo = clamp_lo;
@@ -281,7 +288,7 @@ Problem make_ex(const void* A, const void* B, const void* bias, const void* R, i
 
 bool bad(const Problem& p) {
   return !p.A || !p.B || p.M < 1 || p.N < 1 || p.K < 1 || p.batch < 1 || p.act < 0 || p.act > ACT_LAST ||
-         (p.beta != 0.0 && !p.R);
+         (p.beta != 0.0 && !p.R) || (p.a_symmetric && p.M != p.K);
 }
 
 }  // namespace

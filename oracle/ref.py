@@ -23,6 +23,7 @@ FLAG_BIAS_PER_ROW = 1 << 10
 FLAG_B_BROADCAST = 1 << 11
 FLAG_CLAMP = 1 << 12
 FLAG_IN_F32 = 1 << 13
+FLAG_A_SYMMETRIC = 1 << 14      # extended entry points: A is square and symmetric, its upper triangle is the matrix
 OUT_BF16, OUT_F16, OUT_F32 = 0, 1, 2
 REDUCE_SUM, REDUCE_MAX, REDUCE_LOGSUMEXP = 1, 2, 3
 
@@ -156,7 +157,8 @@ def gemm_epilogue_points(A, B, bias, R, idx, M, N, K, batch, alpha, beta, act):
 def gemm_epilogue_ex(A, B, bias, R, M, N, K, batch, alpha, beta, act, row_scale=None, col_scale=None, clamp_lo=0.0,
                      clamp_hi=0.0, out_dtype=OUT_BF16, rows=None):
     """Extended consumer family: scale vectors, per-row bias, clamp, shared B, bf16 / fp16 / fp32 output,
-    and (FLAG_IN_F32) float32 operands multiplied as TF32.
+    (FLAG_IN_F32) float32 operands multiplied as TF32, and (FLAG_A_SYMMETRIC) a square symmetric A given by its
+    upper triangle (what the array holds below the diagonal is ignored).
     Returns (D64, Dout) for the whole problem ([batch,M,N]) or for ``rows`` ([len(rows),N]); Dout is
     uint16 bit patterns (bf16, fp16) or float32."""
     in_dtype = np.float32 if act & FLAG_IN_F32 else np.uint16

@@ -303,3 +303,59 @@ def test_row_reduction_large_values_do_not_overflow(oracle):
     lse = run_reduce(oracle, p, oracle.REDUCE_LOGSUMEXP)[2]
     b = p.bias.astype(np.float64)
     assert np.all(np.isfinite(lse)) and np.allclose(lse, b.max() + np.log(np.exp(b - b.max()).sum()), rtol=1e-15)
+
+
+# ---------------------------------------------------------------- symmetric A (the GEMM prompt's structure hint)
+
+def test_symmetric_flag_is_a_no_op_on_a_symmetric_matrix(oracle):
+    p = W.make(40, 24, 40, batch=2, seed=9, act=W.ACT_SILU | W.FLAG_A_SYMMETRIC, A=("normal", 1.0), B=("normal", 0.3),
+               bias=("normal", 1.0))
+    assert np.array_equal(p.A, p.A.transpose(0, 2, 1))
+    s64, s16 = run_ex(oracle, p)
+    plain = p.act & ~W.FLAG_A_SYMMETRIC
+    b64, b16 = oracle.gemm_epilogue(p.A, p.B, p.bias, p.R, p.M, p.N, p.K, p.batch, p.alpha, p.beta, plain)
+    assert np.array_equal(s64, b64) and np.array_equal(s16, b16)
+
+
+def test_symmetric_flag_never_looks_below_the_diagonal(oracle):
+    """NaNs below the diagonal change nothing, and the result is numpy's fp64 product with the mirrored matrix."""
+    m = 40
+    p = W.make(m, 16, m, batch=2, seed=10, act=W.FLAG_A_SYMMETRIC, A=("normal", 1.0), B=("normal", 1.0))
+    a = W.poison_below_blocks(p.A, 1)                       # every element below the diagonal is a NaN
+    assert np.isnan(f64(a)[:, 5, 2]).all() and not np.isnan(f64(a)[:, 2, 5]).any()
+    d64, _ = oracle.gemm_epilogue_ex(a, p.B, None, None, m, 16, m, 2, 1.0, 0.0, p.act)
+    upper = np.triu(f64(p.A))
+    full = upper + np.triu(f64(p.A), 1).transpose(0, 2, 1)
+    assert np.allclose(d64, full @ f64(p.B), rtol=1e-13, atol=1e-13)
+
+
+def test_symmetric_flag_closed_forms(oracle):
+    m, n = 24, 8
+    ones, zero = gen.f32_to_bf16_bits(np.float32(1.0)), np.uint16(0)
+    a = np.where(np.triu(np.ones((m, m), dtype=bool)), ones, zero).astype(np.uint16)[None]     # upper triangle of ones
+    b = np.full((1, m, n), ones, dtype=np.uint16)
+    d_sym, _ = oracle.gemm_epilogue_ex(a, b, None, None, m, n, m, 1, 1.0, 0.0, W.FLAG_A_SYMMETRIC)
+    d_tri, _ = oracle.gemm_epilogue_ex(a, b, None, None, m, n, m, 1, 1.0, 0.0, 0)
+    assert np.array_equal(d_sym, np.full((1, m, n), float(m)))                   # the mirrored matrix is all ones
+    assert np.array_equal(d_tri[0, :, 0], m - np.arange(m, dtype=np.float64))    # the stored one is triangular
+    # A[i,k] = 16 i + k above the diagonal, identity B: D[i,j] = 16 min(i,j) + max(i,j)
+    m = 16
+    i, k = np.meshgrid(np.arange(m), np.arange(m), indexing="ij")
+    a = gen.f32_to_bf16_bits(np.where(k >= i, 16 * i + k, -1).astype(np.float32))[None]
+    eye = gen.f32_to_bf16_bits(np.eye(m, dtype=np.float32))[None]
+    d, _ = oracle.gemm_epilogue_ex(a, eye, None, None, m, m, m, 1, 1.0, 0.0, W.FLAG_A_SYMMETRIC)
+    assert np.array_equal(d[0], (16 * np.minimum(i, k) + np.maximum(i, k)).astype(np.float64))
+
+
+def test_symmetric_flag_needs_a_square_matrix(oracle):
+    p = W.make(16, 8, 24, seed=1)
+    with pytest.raises(ValueError):
+        oracle.gemm_epilogue_ex(p.A, p.B, None, None, 16, 8, 24, 1, 1.0, 0.0, W.FLAG_A_SYMMETRIC)
+
+
+def test_symmetric_flag_reaches_the_row_reduction(oracle):
+    p = W.make(24, 16, 24, seed=11, act=W.FLAG_A_SYMMETRIC, A=("smallint", 1.0), B=("smallint", 1.0))
+    a = W.poison_below_blocks(p.A, 1)
+    d64, _ = oracle.gemm_epilogue_ex(a, p.B, None, None, 24, 16, 24, 1, 1.0, 0.0, p.act)
+    out = oracle.gemm_epilogue_reduce(a, p.B, None, None, 24, 16, 24, 1, 1.0, 0.0, p.act, 1)
+    assert np.array_equal(out[-1].reshape(-1), d64.sum(axis=-1).reshape(-1))
