@@ -465,6 +465,47 @@ def conv_row(ctx, device, peaks, flush):
             "torch_conv_bias_relu_us_best": min(tl) * 1e6, "torch_conv_only_us_best": min(tlo) * 1e6, "plan": plan}
 
 
+def symm_rows(ctx, device, peaks, flush):
+    """Symmetric A (CG_FLAG_A_SYMMETRIC) against the same call without the flag, on a memory-bound shape -- an
+    8192 x 8192 symmetric A (134 MB) times a 128-column B -- and on the compute-bound 4096-cube; + bias + SiLU.
+    Algorithmic bytes with the flag: the upper triangle of A (diagonal blocks whole), B, bias, D."""
+    import torch
+    out = {}
+    for m, n in ((8192, 128), (4096, 4096)):
+        g = torch.Generator(device=device)
+        g.manual_seed(7)
+        a = torch.randn((m, m), device=device, generator=g)
+        a = (torch.triu(a) + torch.triu(a, 1).t()).to(torch.bfloat16).contiguous()
+        b = (torch.randn((n, m), device=device, generator=g) * (1.0 / 64.0)).to(torch.bfloat16)       # [N, K]
+        bias = torch.randn((n,), device=device, generator=g)
+        d = torch.empty((m, n), device=device, dtype=torch.bfloat16)
+        act = W.ACT_SILU | W.FLAG_B_COLMAJOR
+        row = {}
+        for label, flag in (("symmetric", W.FLAG_A_SYMMETRIC), ("plain", 0)):
+            call = lambda: ctx.gemm_epilogue_ex(a, b, bias, None, d, m, n, m, 1, 1.0, 0.0, act | flag)
+            timed(call, 3, flush)
+            ts = timed(call, 10, flush)
+            ctx.check()
+            row[f"{label}_us_best"] = min(ts) * 1e6
+            row[f"{label}_us_median"] = float(np.median(ts)) * 1e6
+            row[f"{label}_plan"] = ctx.last_plan()
+        lib = lambda: torch.matmul(a, b.t(), out=d)
+        timed(lib, 3, flush)
+        row["cublas_gemm_only_us_best"] = min(timed(lib, 10, flush)) * 1e6
+        flops = 2.0 * m * m * n
+        bytes_plain = 2.0 * (m * m + m * n + m * n) + 4.0 * n
+        bytes_symm = bytes_plain - 2.0 * (m * m - m * 256) / 2.0              # what lies below the 256-wide diagonal band is not read
+        best = row["symmetric_us_best"] * 1e-6
+        row.update({"workload": f"symmetric A {m} x {m} bf16, B [{n}, {m}] (K-major), bias fp32, SiLU", "flops": flops,
+                    "algorithmic_bytes_plain": bytes_plain, "algorithmic_bytes_symmetric": bytes_symm,
+                    "tflops_best": flops / best / 1e12, "gbs_best_of_symmetric_bytes": bytes_symm / best / 1e9,
+                    "gbs_equivalent_of_plain_bytes": bytes_plain / best / 1e9,
+                    "frac_hbm_of_measured": bytes_symm / best / 1e9 / peaks["hbm_gbs"],
+                    "frac_tensor_of_measured_burst": flops / best / 1e12 / peaks["bf16_tflops"]})
+        out[f"{m}x{n}"] = row
+    return out
+
+
 def workload_table(ctx, device, peaks, names):
     """All five workloads under the heuristic plan, each launch timed alone after an L2 flush (their
     inputs may fit in L2)."""
@@ -498,6 +539,7 @@ def workload_table(ctx, device, peaks, names):
         out["next_tf32_8192"] = tf32_row(ctx, device, peaks, flush)
         out["next_diag_matmul_8192"] = diag_rows(ctx, device, peaks, flush)
         out["next_conv3x3_256"] = conv_row(ctx, device, peaks, flush)
+        out["next_symmetric_a"] = symm_rows(ctx, device, peaks, flush)
     return out
 
 
@@ -629,7 +671,7 @@ def run_row(args):
     device = torch.device("cuda", 0)
     ctx = cg.Context(0)
     flush = L2Flush(device)
-    fn = {"tf32": tf32_row, "diag": diag_rows, "conv": conv_row}[args.row]
+    fn = {"tf32": tf32_row, "diag": diag_rows, "conv": conv_row, "symm": symm_rows}[args.row]
     row = fn(ctx, device, load_peaks(), flush)
     print(json.dumps({"row": args.row, "result": row}), flush=True)
 
@@ -644,7 +686,7 @@ def main():
     ap.add_argument("--no-table", action="store_true", help="skip the five-workload table")
     for flag in ("tile-n", "cta-group", "num-units", "dp-units", "stages", "group-m", "max-ctas"):
         ap.add_argument(f"--{flag}", type=int, default=0, help="plan override for ablations (0 = heuristic)")
-    ap.add_argument("--row", choices=["tf32", "diag", "conv"], default=None,
+    ap.add_argument("--row", choices=["tf32", "diag", "conv", "symm"], default=None,
                     help="only that row of the 'next' part of the table (a few launches; for profiler runs)")
     ap.add_argument("--kernel-only", action="store_true",
                     help="only the device-timed region (for profiler runs): no e2e, no CPU baseline, no table")

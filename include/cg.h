@@ -108,6 +108,15 @@ CG_API int cg_gemm_epilogue(cg_handle_t h, const void* A, const void* B, const v
  *                         paper's square-GEMM case study): the tensor core drops the 13 low fraction bits of each
  *                         operand.  B must be stored [batch,N,K] (CG_FLAG_B_COLMAJOR, else CG_ERR_UNSUPPORTED);
  *                         K % 4 == 0 would do for the fp32 row pitch, K % 8 == 0 is still required
+ *   CG_FLAG_A_SYMMETRIC   A is square (M == K, else CG_ERR_INVALID_ARG) and symmetric in every batch entry (the GEMM
+ *                         prompt's hint: "if a matrix is symmetric the number of reads could be reduced").  The
+ *                         caller vouches for the symmetry; the kernel then fetches only the 64-column blocks that
+ *                         lie on or above the tile's diagonal block and takes every block to the left of it from
+ *                         its mirror image above the diagonal, so that each block above the diagonal serves two
+ *                         row tiles and the second use hits in L2.  Elements below the diagonal are read only
+ *                         inside the 256 x 256 squares on the diagonal; everything else there may hold anything.
+ *                         bf16 operands only (with CG_FLAG_IN_F32: CG_ERR_UNSUPPORTED); tile shapes 128 x 128,
+ *                         128 x 256 and the 256 x 256 pair tile (another forced shape: CG_ERR_INVALID_ARG)
  * and in *ex (NULL = all off, the call then equals cg_gemm_epilogue):
  *   row_scale, col_scale  device, fp32 [M] / [N], or NULL (= 1); they scale the product like alpha, never the bias;
  *                         shared by all batch entries
@@ -124,7 +133,8 @@ CG_API int cg_gemm_epilogue(cg_handle_t h, const void* A, const void* B, const v
  * Errors as for cg_gemm_epilogue; CG_ERR_INVALID_ARG also for clamp_lo > clamp_hi, CG_FLAG_CLAMP without ex, an
  * unknown row_reduce code or a reduction without row_out.
  */
-enum { CG_FLAG_BIAS_PER_ROW = 1 << 10, CG_FLAG_B_BROADCAST = 1 << 11, CG_FLAG_CLAMP = 1 << 12, CG_FLAG_IN_F32 = 1 << 13 };
+enum { CG_FLAG_BIAS_PER_ROW = 1 << 10, CG_FLAG_B_BROADCAST = 1 << 11, CG_FLAG_CLAMP = 1 << 12, CG_FLAG_IN_F32 = 1 << 13,
+       CG_FLAG_A_SYMMETRIC = 1 << 14 };
 enum { CG_OUT_BF16 = 0, CG_OUT_F16 = 1, CG_OUT_F32 = 2 };
 enum { CG_REDUCE_NONE = 0, CG_REDUCE_SUM = 1, CG_REDUCE_MAX = 2, CG_REDUCE_LOGSUMEXP = 3 };
 typedef struct cg_epilogue_ex {

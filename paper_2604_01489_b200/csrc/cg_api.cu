@@ -135,22 +135,28 @@ struct KernelEntry {
   int stage_bytes, fixed_bytes, r_bytes, stages_max, stages_max_r, threads, sub_cols;
 };
 
-template <int BN, int CGN, bool KM, bool CONV = false>
+template <int BN, int CGN, bool KM, int MODE = MODE_GEMM>
 KernelEntry entry() {
   using C = Cfg<BN, CGN, KM>;
-  return KernelEntry{gemm_epilogue_kernel<BN, CGN, KM, CONV>, C::STAGE_BYTES, C::FIXED_BYTES, C::R_BYTES, C::stages_max(false),
+  return KernelEntry{gemm_epilogue_kernel<BN, CGN, KM, MODE>, C::STAGE_BYTES, C::FIXED_BYTES, C::R_BYTES, C::stages_max(false),
                      C::stages_max(true), C::NUM_THREADS, C::SUB_COLS};
 }
 
 // index: [bn_idx (64,128,256)][cg-1][b_kmajor]
-bool lookup(int bn, int cgn, bool km, KernelEntry* out, bool conv = false) {
-  if (conv) {                 // the convolution instances: K-major weights, rank-4 maps for the image and the output
-    if (cgn == 1 && bn == 64) { *out = entry<64, 1, true, true>(); return true; }
-    if (cgn == 1 && bn == 128) { *out = entry<128, 1, true, true>(); return true; }
-    if (cgn == 1 && bn == 256) { *out = entry<256, 1, true, true>(); return true; }
-    if (cgn == 2 && bn == 128) { *out = entry<128, 2, true, true>(); return true; }
-    if (cgn == 2 && bn == 256) { *out = entry<256, 2, true, true>(); return true; }
-    if (cgn == 2 && bn == 512) { *out = entry<512, 2, true, true>(); return true; }
+bool lookup(int bn, int cgn, bool km, KernelEntry* out, int mode = MODE_GEMM) {
+  if (mode == MODE_CONV) {    // the convolution instances: K-major weights, rank-4 maps for the image and the output
+    if (cgn == 1 && bn == 64) { *out = entry<64, 1, true, MODE_CONV>(); return true; }
+    if (cgn == 1 && bn == 128) { *out = entry<128, 1, true, MODE_CONV>(); return true; }
+    if (cgn == 1 && bn == 256) { *out = entry<256, 1, true, MODE_CONV>(); return true; }
+    if (cgn == 2 && bn == 128) { *out = entry<128, 2, true, MODE_CONV>(); return true; }
+    if (cgn == 2 && bn == 256) { *out = entry<256, 2, true, MODE_CONV>(); return true; }
+    if (cgn == 2 && bn == 512) { *out = entry<512, 2, true, MODE_CONV>(); return true; }
+    return false;
+  }
+  if (mode == MODE_SYMM) {    // symmetric A: three tile shapes (see make_plan)
+    if (cgn == 1 && bn == 128) { *out = km ? entry<128, 1, true, MODE_SYMM>() : entry<128, 1, false, MODE_SYMM>(); return true; }
+    if (cgn == 1 && bn == 256) { *out = km ? entry<256, 1, true, MODE_SYMM>() : entry<256, 1, false, MODE_SYMM>(); return true; }
+    if (cgn == 2 && bn == 256) { *out = km ? entry<256, 2, true, MODE_SYMM>() : entry<256, 2, false, MODE_SYMM>(); return true; }
     return false;
   }
   if (cgn == 1) {
@@ -188,7 +194,10 @@ int prepare_kernels(cg_context* h) {
         if (!lookup(bns[i], cgn, km != 0, &e)) continue;
         CG_CUDA(h, cudaFuncSetAttribute(reinterpret_cast<const void*>(e.fn), cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         SMEM_LIMIT));
-        if (km != 0 && lookup(bns[i], cgn, true, &e, true))
+        if (km != 0 && lookup(bns[i], cgn, true, &e, MODE_CONV))
+          CG_CUDA(h, cudaFuncSetAttribute(reinterpret_cast<const void*>(e.fn), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          SMEM_LIMIT));
+        if (lookup(bns[i], cgn, km != 0, &e, MODE_SYMM))
           CG_CUDA(h, cudaFuncSetAttribute(reinterpret_cast<const void*>(e.fn), cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           SMEM_LIMIT));
       }
@@ -255,7 +264,7 @@ size_t partial_need(long long split_units, int bn, int cgn) {
 }
 
 int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, bool has_r, Plan* pl, bool r_own_only = false,
-              int bk_elems = BK) {
+              int bk_elems = BK, int mode = MODE_GEMM) {
   const cg_tuning_t& t = h->tuning;
   const int sms = (t.max_ctas > 0 && t.max_ctas < h->num_sms) ? t.max_ctas : h->num_sms;
   const int k_blocks = ceil_div(K, bk_elems);
@@ -290,6 +299,11 @@ int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, bool
       if (N >= 256 && tiles(BM, 256) >= sms) bn = 256;
     }
   }
+  if (mode == MODE_SYMM) {       // the symmetric form exists for 128- and 256-wide tiles and the 256 x 256 pair tile
+    if (cgn == 2 && bn == 128 && t.tile_n == 0) cgn = 1;
+    if (bn == 64 && t.tile_n == 0) bn = 128;
+    if (bn == 512 && t.tile_n == 0) bn = 256;
+  }
   // Problems of under one wave of 1-CTA tiles: split K across the CTAs of a cluster, which exchange
   // their partial tiles through distributed shared memory.  Wider tiles first (an MMA costs the same
   // whatever its N, and more of B is in flight per SM); each CTA must own at least 64 columns.
@@ -314,7 +328,8 @@ int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, bool
     }
   }
   KernelEntry e;
-  if (!lookup(bn, cgn, b_kmajor, &e)) return fail(h, CG_ERR_INVALID_ARG, "no kernel for tile_n=%d cta_group=%d", bn, cgn);
+  if (!lookup(bn, cgn, b_kmajor, &e, mode == MODE_SYMM ? MODE_SYMM : MODE_GEMM))
+    return fail(h, CG_ERR_INVALID_ARG, "no kernel for tile_n=%d cta_group=%d%s", bn, cgn, mode == MODE_SYMM ? " with a symmetric A" : "");
 
   pl->bn = bn;
   pl->cg = cgn;
@@ -477,7 +492,8 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
            int batch, float alpha, float beta, int act, cudaStream_t stream, const cg_epilogue_ex_t* ex = nullptr,
            const ConvGeom* conv = nullptr) {
   const bool b_kmajor = (act & CG_FLAG_B_COLMAJOR) != 0;
-  const bool ext_in_use = (act & (CG_FLAG_BIAS_PER_ROW | CG_FLAG_B_BROADCAST | CG_FLAG_CLAMP | CG_FLAG_IN_F32)) != 0 ||
+  const bool symm = (act & CG_FLAG_A_SYMMETRIC) != 0;
+  const bool ext_in_use = (act & (CG_FLAG_BIAS_PER_ROW | CG_FLAG_B_BROADCAST | CG_FLAG_CLAMP | CG_FLAG_IN_F32 | CG_FLAG_A_SYMMETRIC)) != 0 ||
                           (ex && (ex->row_scale || ex->col_scale || ex->out_dtype != CG_OUT_BF16 || ex->row_reduce));
   const int row_reduce = ex ? ex->row_reduce : 0;
   const bool store_d = D != nullptr;
@@ -492,13 +508,15 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   const bool tf32 = (act & CG_FLAG_IN_F32) != 0;
   const int bk_elems = tf32 ? BK / 2 : BK;
   const int in_dtype = tf32 ? CG_OUT_F32 : CG_OUT_BF16;           // (element type code of A and B)
-  int rc = make_plan(h, M, N, K, batch, b_kmajor, beta != 0.0f, &pl, out_dtype == CG_OUT_F32 || !store_d, bk_elems);
+  const int mode = conv ? MODE_CONV : (symm ? MODE_SYMM : MODE_GEMM);
+  int rc = make_plan(h, M, N, K, batch, b_kmajor, beta != 0.0f, &pl, out_dtype == CG_OUT_F32 || !store_d, bk_elems, mode);
   if (rc != CG_OK) return rc;
   KernelEntry e;
-  lookup(pl.bn, pl.cg, b_kmajor, &e, conv != nullptr);
+  lookup(pl.bn, pl.cg, b_kmajor, &e, mode);
 
   CUtensorMap tmA, tmB, tmD, tmR;
   if (conv) rc = make_map4(h, &tmA, A, conv->IC, conv->W, conv->H, conv->n_img, BK, CONV_TILE_W, CONV_TILE_H, conv->stride);
+  else if (symm) rc = make_map(h, &tmA, A, K, M, batch, 64, 64);      // serves blocks read as they are and mirrored ones
   else rc = make_map(h, &tmA, A, K, M, batch, bk_elems, BM, in_dtype);
   if (rc != CG_OK) return rc;
   const int b_entries = b_broadcast ? 1 : batch;
@@ -759,10 +777,13 @@ int cg_gemm_epilogue_ex(cg_handle_t h, const void* A, const void* B, const void*
     return fail(h, CG_ERR_INVALID_ARG, "row_reduce must be a CG_REDUCE_* code with a 4-byte aligned row_out");
   // with a row reduction D may be NULL (only the reduction is wanted)
   int rc = validate(h, A, B, bias, R, (!D && reducing) ? const_cast<void*>(A) : D, M, N, K, batch, beta, act,
-                    CG_FLAG_BIAS_PER_ROW | CG_FLAG_B_BROADCAST | CG_FLAG_CLAMP | CG_FLAG_IN_F32);
+                    CG_FLAG_BIAS_PER_ROW | CG_FLAG_B_BROADCAST | CG_FLAG_CLAMP | CG_FLAG_IN_F32 | CG_FLAG_A_SYMMETRIC);
   if (rc != CG_OK) return rc;
   if ((act & CG_FLAG_IN_F32) && !(act & CG_FLAG_B_COLMAJOR))
     return fail(h, CG_ERR_UNSUPPORTED, "fp32 operands need B stored [batch,N,K] (CG_FLAG_B_COLMAJOR)");
+  if ((act & CG_FLAG_A_SYMMETRIC) && M != K) return fail(h, CG_ERR_INVALID_ARG, "a symmetric A is square (got M=%d K=%d)", M, K);
+  if ((act & CG_FLAG_A_SYMMETRIC) && (act & CG_FLAG_IN_F32))
+    return fail(h, CG_ERR_UNSUPPORTED, "the symmetric form exists for bf16 operands only");
   if ((rc = check_alignment(h, A, B, (act & CG_FLAG_BIAS_PER_ROW) ? nullptr : bias, R, D ? D : const_cast<void*>(A), beta, act)) != CG_OK)
     return rc;
   if (ex) {

@@ -6,14 +6,16 @@
 // shared by the batch, fp16 / fp32 output, fp32 operands multiplied as TF32, and a fused reduction of
 // every output row).
 //
-// Roles inside one CTA of 64 + 32 * EPI_WARPS threads (EPI_WARPS = 4 for 64-wide tiles, else 8):
+// Roles inside one CTA of 32 * (LEAD_WARPS + EPI_WARPS) threads (EPI_WARPS = 4 for 64-wide tiles, else 8;
+// LEAD_WARPS = 2, or 4 for the 512-wide tile, whose warps 2 and 3 only complete the first warpgroup so
+// that it can hand registers to the epilogue warpgroups):
 //   warp 0 (one lane)  producer: TMA loads of A and B k-blocks into an N-stage shared-memory
 //                      ring, completion counted in bytes on `full[stage]` mbarriers;
 //   warp 1 (one lane)  MMA issuer: tcgen05.mma (bf16 x bf16 or TF32 x TF32 -> fp32) from the ring into
 //                      an accumulator buffer in tensor memory; tcgen05.commit frees ring stages
 //                      (`empty[stage]`) and publishes accumulators (`acc_full[buf]`); the whole
 //                      warp allocates / frees tensor memory;
-//   warps 2 and up     epilogue: TMEM -> registers, alpha*acc + bias, activation, + beta*R,
+//   the other warps    epilogue: TMEM -> registers, alpha*acc + bias, activation, + beta*R,
 //                      rounding, swizzled shared-memory staging, TMA store.  D is written once and
 //                      never read.  A warp owns the 32 accumulator rows (TMEM lanes) of its quarter
 //                      and, with eight warps, one half of the tile's columns; it never synchronises
@@ -28,6 +30,11 @@
 // split-K / stream-K: every contributor writes its fp32 partial to the workspace,
 // draws a ticket, and the last one to arrive sums all partials in unit order (deterministic)
 // and runs the epilogue.  Nobody ever waits for another CTA.
+//
+// MODE (template parameter) says what A is: a matrix (rank-3 map), an NHWC image read through rank-4
+// boxes (convolution as an implicit GEMM), or a square symmetric matrix of which only the blocks on or
+// above the diagonal are fetched (a block left of the diagonal comes from its mirror image and is
+// multiplied as an M-major operand).
 //
 // With CG == 2 a pair of CTAs (cluster 2x1) shares one 256 x BN tile: each CTA loads its own
 // 128 rows of A and half of the B columns, the leader CTA issues tcgen05.mma.cta_group::2,
@@ -87,6 +94,7 @@ struct ConvGeom {
   int tiles_h, tiles_w;   // pixel tiles per image
 };
 constexpr int CONV_TILE_H = 8, CONV_TILE_W = 16;
+enum { MODE_GEMM = 0, MODE_CONV = 1, MODE_SYMM = 2 };    // what the A operand is (a template parameter of the kernel)
 
 struct KernelParams {
   int M, N, K, batch;
@@ -175,6 +183,7 @@ struct Cfg {
   static constexpr int TMEM_COLS = ACC_BUFS * BN <= 32 ? 32 : (ACC_BUFS * BN <= 64 ? 64 : (ACC_BUFS * BN <= 128 ? 128 : (ACC_BUFS * BN <= 256 ? 256 : 512)));
   static constexpr uint32_t IDESC = ptx::instr_desc_bf16(BM * CG, MMA_N, !B_KMAJOR);
   static constexpr uint32_t IDESC_TF32 = ptx::instr_desc_tf32(BM * CG, MMA_N);
+  static constexpr uint32_t IDESC_A_MIRRORED = IDESC | ptx::INSTR_DESC_A_MN_MAJOR;   // A read M-major (symmetric A, mirrored block)
   __host__ __device__ static constexpr int layout_bytes(int stages, bool with_r) {
     return stages * STAGE_BYTES + FIXED_BYTES + (with_r ? R_BYTES : 0);
   }
@@ -439,12 +448,14 @@ __device__ __forceinline__ void stage_chunk(const uint32_t (&out)[EPI_COLS / 2],
 
 // ---------------------------------------------------------------- the kernel
 
-template <int BN, int CG, bool B_KMAJOR, bool CONV = false>
+template <int BN, int CG, bool B_KMAJOR, int MODE = MODE_GEMM>
 __global__ void __launch_bounds__((Cfg<BN, CG, B_KMAJOR>::NUM_THREADS), 1)
 gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                      const __grid_constant__ CUtensorMap tmD, const __grid_constant__ CUtensorMap tmR,
                      const KernelParams p) {
   using C = Cfg<BN, CG, B_KMAJOR>;
+  constexpr bool CONV = (MODE == MODE_CONV);     // A is an NHWC image read through rank-4 boxes
+  constexpr bool SYMM = (MODE == MODE_SYMM);     // A is square and symmetric: only blocks on or above the diagonal are read
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = ptx::smem_u32(smem_raw);
   const uint32_t pad = ((raw_addr + 1023u) & ~1023u) - raw_addr;
@@ -488,6 +499,16 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       if (!withhold_a) ptx::tma_load_4d(a_dst, &tmA, bar, icb * BK, w0 * p.cv.stride - p.cv.pad_w + kw * p.cv.dilation,
                                         h0 * p.cv.stride - p.cv.pad_h + kh * p.cv.dilation, n);
       k0 = tap * p.cv.IC + icb * BK;                   // the weights' K index of this block
+    } else if constexpr (SYMM) {
+      // Symmetric A through 64 x 64 boxes.  A k-block left of the tile's diagonal block is fetched from its
+      // mirror image above the diagonal -- rows k0.., columns m0.. -- and lands M-major (64 k-rows of 128
+      // bytes per 64 rows of the tile), which the MMA reads through the transposed operand form.
+      const bool mirrored = k0 + BK <= m0;
+#pragma unroll
+      for (int j = 0; j < BM / 64; ++j) {
+        if (mirrored) ptx::tma_load_3d(a_dst + j * (64 * BK * 2), &tmA, bar, m0 + j * 64, k0, b);
+        else ptx::tma_load_3d(a_dst + j * (64 * BK * 2), &tmA, bar, k0, m0 + j * 64, b);
+      }
     } else if (!withhold_a) {
       ptx::tma_load_3d(a_dst, &tmA, bar, k0, m0, b);   // (withheld only by the starvation test hook)
     }
@@ -577,6 +598,13 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
               ptx::tma_load_4d_pair(a_dst, &tmA, bar, icb * BK, w0 * p.cv.stride - p.cv.pad_w + kw * p.cv.dilation,
                                     h0 * p.cv.stride - p.cv.pad_h + kh * p.cv.dilation, n);
               k0 = tap * p.cv.IC + icb * BK;
+            } else if constexpr (SYMM) {
+              const bool mirrored = k0 + BK <= mt * (BM * CG);      // one decision for the pair: its MMAs are shared
+#pragma unroll
+              for (int j = 0; j < BM / 64; ++j) {
+                if (mirrored) ptx::tma_load_3d_pair(a_dst + j * (64 * BK * 2), &tmA, bar, m0 + j * 64, k0, b);
+                else ptx::tma_load_3d_pair(a_dst + j * (64 * BK * 2), &tmA, bar, k0, m0 + j * 64, b);
+              }
             } else if (!(p.test_starve && issued == 0)) {
               ptx::tma_load_3d_pair(a_dst, &tmA, bar, k0, m0, b);
             }
@@ -656,34 +684,46 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       constexpr int bk_el = TF32 ? BK / 2 : BK, mma_k_el = TF32 ? UMMA_K / 2 : UMMA_K;   // elements per k-block / per MMA
       int tail_nk = (p.K - last_kb * bk_el + mma_k_el - 1) / mma_k_el;    // 32-byte steps of the last k-block
       if (tail_nk > BK / UMMA_K) tail_nk = BK / UMMA_K;
-      auto mma = [&](uint32_t d, uint64_t a, uint64_t b, uint32_t acc_in) {
-        if constexpr (TF32) ptx::mma_tf32<CG>(d, a, b, C::IDESC_TF32, acc_in); else ptx::mma_f16<CG>(d, a, b, C::IDESC, acc_in);
+      auto mma = [&](uint32_t d, uint64_t a, uint64_t b, uint32_t acc_in, uint32_t idesc) {
+        if constexpr (TF32) ptx::mma_tf32<CG>(d, a, b, C::IDESC_TF32, acc_in); else ptx::mma_f16<CG>(d, a, b, idesc, acc_in);
       };
+      // symmetric A: a mirrored k-block is an M-major operand (same form as a row-major B block)
+      const uint32_t a_lo0_mirrored = static_cast<uint32_t>(ptx::smem_desc_sw128(ring_addr, 64 * BK * 2, 8 * 128));
+      constexpr uint32_t A_KSTEP_MIRRORED = (UMMA_K * 128) >> 4;         // +16 k-rows
       auto desc = [&](uint32_t lo) -> uint64_t { return (static_cast<uint64_t>(desc_hi) << 32) | lo; };
       while (ok && wi.next(s)) {
         if (!wait_bar(ptx::smem_u32(&ctrl->acc_empty[acc]), acc_phase ^ 1u, ctrl, p)) { ok = false; break; }
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
         uint32_t accumulate = 0;
+        int tile_row0 = 0;                       // symmetric A: first row of this (pair) tile
+        if constexpr (SYMM) {
+          int tb, tmt, tnt;
+          decode_tile(p, s.tile, tb, tmt, tnt);
+          tile_row0 = tmt * (BM * CG);
+        }
         for (int kb = s.kb0; kb < s.kb1; ++kb) {
           if (!wait_bar(full0 + stage * 8, phase, ctrl, p)) { ok = false; break; }
           if (accumulate == 0 && acc == 0 && acc_phase == 0) trace_event(p, TR_FIRST_FULL);
           ptx::tc_fence_after();
-          const uint32_t a_lo = a_lo0 + stage * STAGE_STEP;
+          const bool mirrored = SYMM && (kb + 1) * BK <= tile_row0;
+          const uint32_t a_lo = (mirrored ? a_lo0_mirrored : a_lo0) + stage * STAGE_STEP;
+          const uint32_t a_kstep = mirrored ? A_KSTEP_MIRRORED : A_KSTEP;
+          const uint32_t idesc = mirrored ? C::IDESC_A_MIRRORED : C::IDESC;
           const uint32_t b_lo = b_lo0 + stage * STAGE_STEP;
           if (kb != last_kb || tail_nk == BK / UMMA_K) {
 #pragma unroll
             for (int k = 0; k < BK / UMMA_K; ++k)
 #pragma unroll
               for (int h = 0; h < C::NSUB; ++h)
-                mma(d_tmem + h * C::MMA_N, desc(a_lo + k * A_KSTEP), desc(b_lo + k * B_KSTEP + h * SUB_STEP),
-                    k == 0 ? accumulate : 1u);
+                mma(d_tmem + h * C::MMA_N, desc(a_lo + k * a_kstep), desc(b_lo + k * B_KSTEP + h * SUB_STEP),
+                    k == 0 ? accumulate : 1u, idesc);
           } else {
             for (int k = 0; k < tail_nk; ++k)     // K tail: skip 16-wide steps that are all padding
 #pragma unroll
               for (int h = 0; h < C::NSUB; ++h)
-                mma(d_tmem + h * C::MMA_N, desc(a_lo + k * A_KSTEP), desc(b_lo + k * B_KSTEP + h * SUB_STEP),
-                    (k > 0) ? 1u : accumulate);
+                mma(d_tmem + h * C::MMA_N, desc(a_lo + k * a_kstep), desc(b_lo + k * B_KSTEP + h * SUB_STEP),
+                    (k > 0) ? 1u : accumulate, idesc);
           }
           accumulate = 1u;
           ptx::tc_commit<CG>(empty0 + stage * 8);

@@ -276,6 +276,8 @@ __host__ __device__ constexpr uint32_t instr_desc_bf16(int m, int n, bool b_mn_m
          (static_cast<uint32_t>(m >> 4) << 24);
 }
 
+constexpr uint32_t INSTR_DESC_A_MN_MAJOR = 1u << 15;     // A operand stored M-major ("transposed") instead of K-major
+
 // Instruction descriptor, kind::tf32: as above with TF32 A and B (format code 2), both K-major.
 __host__ __device__ constexpr uint32_t instr_desc_tf32(int m, int n) {
   return (1u << 4) | (2u << 7) | (2u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(m >> 4) << 24);
