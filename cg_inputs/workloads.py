@@ -27,6 +27,7 @@ FLAG_B_BROADCAST = 1 << 11
 FLAG_CLAMP = 1 << 12
 FLAG_IN_F32 = 1 << 13
 FLAG_A_SYMMETRIC = 1 << 14
+FLAG_B_SYMMETRIC = 1 << 15
 OUT_BF16, OUT_F16, OUT_F32 = 0, 1, 2
 
 
@@ -55,7 +56,7 @@ class Problem:
 
     @property
     def extended(self) -> bool:
-        return bool(self.act & (FLAG_BIAS_PER_ROW | FLAG_B_BROADCAST | FLAG_CLAMP | FLAG_IN_F32 | FLAG_A_SYMMETRIC)) or self.row_scale is not None \
+        return bool(self.act & (FLAG_BIAS_PER_ROW | FLAG_B_BROADCAST | FLAG_CLAMP | FLAG_IN_F32 | FLAG_A_SYMMETRIC | FLAG_B_SYMMETRIC)) or self.row_scale is not None \
             or self.col_scale is not None or self.out_dtype != OUT_BF16
 
     @property
@@ -116,6 +117,11 @@ def make(M, N, K, batch=1, seed=0, act=ACT_NONE, alpha=1.0, beta=0.0, A=("unifor
         a[:, iu[1], iu[0]] = a[:, iu[0], iu[1]]
     b = gen.tensor(seed, gen.TENSOR_B, (1 if act & FLAG_B_BROADCAST else batch, K, N), B[0], B[1], dtype=in_dtype,
                    colmajor_last2=colmajor)
+    if act & FLAG_B_SYMMETRIC:
+        if N != K:
+            raise ValueError("a symmetric B is square")
+        iu = np.triu_indices(N, 1)
+        b[:, iu[1], iu[0]] = b[:, iu[0], iu[1]]
     bias_arr = None
     if bias is not None:
         want = "bf16" if act & FLAG_BIAS_BF16 else "f32"

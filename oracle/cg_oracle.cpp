@@ -99,7 +99,7 @@ enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU_TANH = 2, ACT_SILU = 3,
 constexpr int ACT_LAST = ACT_LEAKY_RELU;
 constexpr double LEAKY_SLOPE = 0.01;
 enum { FLAG_B_COLMAJOR = 1 << 8, FLAG_BIAS_BF16 = 1 << 9, FLAG_BIAS_PER_ROW = 1 << 10, FLAG_B_BROADCAST = 1 << 11,
-       FLAG_CLAMP = 1 << 12, FLAG_IN_F32 = 1 << 13, FLAG_A_SYMMETRIC = 1 << 14 };
+       FLAG_CLAMP = 1 << 12, FLAG_IN_F32 = 1 << 13, FLAG_A_SYMMETRIC = 1 << 14, FLAG_B_SYMMETRIC = 1 << 15 };
 enum { OUT_BF16 = 0, OUT_F16 = 1, OUT_F32 = 2 };
 enum { REDUCE_NONE = 0, REDUCE_SUM = 1, REDUCE_MAX = 2, REDUCE_LOGSUMEXP = 3 };
 
@@ -168,7 +168,7 @@ struct Problem {
   int act;
   bool b_colmajor, bias_bf16;
   // extended family (all off in the base entry points)
-  bool bias_per_row = false, b_broadcast = false, clamp = false, in_f32 = false, a_symmetric = false;
+  bool bias_per_row = false, b_broadcast = false, clamp = false, in_f32 = false, a_symmetric = false, b_symmetric = false;
   const float* row_scale = nullptr;   // [M] or null
   const float* col_scale = nullptr;   // [N] or null
   double clamp_lo = 0.0, clamp_hi = 0.0;
@@ -198,8 +198,11 @@ inline double a_at(const Problem& p, int64_t b, int64_t m, int64_t k) {
 
 // B[b,k,n] through an index function: row-major [batch,K,N] or column-major [batch,N,K];
 // a shared B has a single batch entry.
+// Under the symmetric flag B is square and the upper triangle of the stored array is the matrix, whichever
+// layout flag is given (a symmetric matrix is its own transpose).
 inline double b_at(const Problem& p, int64_t b, int64_t k, int64_t n) {
   const int64_t base = (p.b_broadcast ? 0 : b) * p.K * p.N;
+  if (p.b_symmetric) return operand(p, p.B, base + (k < n ? k * p.N + n : n * p.N + k));
   return operand(p, p.B, p.b_colmajor ? base + n * p.K + k : base + k * p.N + n);
 }
 
@@ -278,6 +281,7 @@ Problem make_ex(const void* A, const void* B, const void* bias, const void* R, i
   p.clamp = (act & FLAG_CLAMP) != 0;
   p.in_f32 = (act & FLAG_IN_F32) != 0;
   p.a_symmetric = (act & FLAG_A_SYMMETRIC) != 0;
+  p.b_symmetric = (act & FLAG_B_SYMMETRIC) != 0;
   p.row_scale = row_scale;
   p.col_scale = col_scale;
   p.clamp_lo = clamp_lo;
@@ -288,7 +292,7 @@ Problem make_ex(const void* A, const void* B, const void* bias, const void* R, i
 
 bool bad(const Problem& p) {
   return !p.A || !p.B || p.M < 1 || p.N < 1 || p.K < 1 || p.batch < 1 || p.act < 0 || p.act > ACT_LAST ||
-         (p.beta != 0.0 && !p.R) || (p.a_symmetric && p.M != p.K);
+         (p.beta != 0.0 && !p.R) || (p.a_symmetric && p.M != p.K) || (p.b_symmetric && p.N != p.K);
 }
 
 }  // namespace

@@ -24,6 +24,7 @@ FLAG_B_BROADCAST = 1 << 11
 FLAG_CLAMP = 1 << 12
 FLAG_IN_F32 = 1 << 13
 FLAG_A_SYMMETRIC = 1 << 14      # extended entry points: A is square and symmetric, its upper triangle is the matrix
+FLAG_B_SYMMETRIC = 1 << 15      # the same for B (N == K; the layout flag is then immaterial)
 OUT_BF16, OUT_F16, OUT_F32 = 0, 1, 2
 REDUCE_SUM, REDUCE_MAX, REDUCE_LOGSUMEXP = 1, 2, 3
 

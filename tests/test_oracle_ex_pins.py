@@ -359,3 +359,37 @@ def test_symmetric_flag_reaches_the_row_reduction(oracle):
     d64, _ = oracle.gemm_epilogue_ex(a, p.B, None, None, 24, 16, 24, 1, 1.0, 0.0, p.act)
     out = oracle.gemm_epilogue_reduce(a, p.B, None, None, 24, 16, 24, 1, 1.0, 0.0, p.act, 1)
     assert np.array_equal(out[-1].reshape(-1), d64.sum(axis=-1).reshape(-1))
+
+
+# ---------------------------------------------------------------- symmetric B
+
+@pytest.mark.parametrize("colmajor", [0, W.FLAG_B_COLMAJOR])
+def test_symmetric_b_flag_is_a_no_op_on_a_symmetric_matrix(oracle, colmajor):
+    p = W.make(24, 40, 40, batch=2, seed=12, act=W.ACT_SILU | W.FLAG_B_SYMMETRIC | colmajor, A=("normal", 1.0),
+               B=("normal", 0.3), bias=("normal", 1.0))
+    assert np.array_equal(p.B, p.B.transpose(0, 2, 1))
+    s64, s16 = run_ex(oracle, p)
+    b64, b16 = oracle.gemm_epilogue(p.A, p.B, p.bias, p.R, p.M, p.N, p.K, p.batch, p.alpha, p.beta, p.act & ~W.FLAG_B_SYMMETRIC)
+    assert np.array_equal(s64, b64) and np.array_equal(s16, b16)
+
+
+@pytest.mark.parametrize("colmajor", [0, W.FLAG_B_COLMAJOR])
+def test_symmetric_b_flag_never_looks_below_the_diagonal(oracle, colmajor):
+    n = 40
+    p = W.make(16, n, n, batch=2, seed=13, act=W.FLAG_B_SYMMETRIC | colmajor, A=("normal", 1.0), B=("normal", 1.0))
+    b = W.poison_below_blocks(p.B, 1)
+    d64, _ = oracle.gemm_epilogue_ex(p.A, b, None, None, 16, n, n, 2, 1.0, 0.0, p.act)
+    full = np.triu(f64(p.B)) + np.triu(f64(p.B), 1).transpose(0, 2, 1)
+    assert np.allclose(d64, f64(p.A) @ full, rtol=1e-13, atol=1e-13)
+
+
+def test_symmetric_b_flag_closed_forms(oracle):
+    n = 16
+    i, k = np.meshgrid(np.arange(n), np.arange(n), indexing="ij")
+    b = gen.f32_to_bf16_bits(np.where(k >= i, 16 * i + k, -1).astype(np.float32))[None]       # stored upper triangle
+    eye = gen.f32_to_bf16_bits(np.eye(n, dtype=np.float32))[None]
+    d, _ = oracle.gemm_epilogue_ex(eye, b, None, None, n, n, n, 1, 1.0, 0.0, W.FLAG_B_SYMMETRIC)
+    assert np.array_equal(d[0], (16 * np.minimum(i, k) + np.maximum(i, k)).astype(np.float64))
+    p = W.make(16, 8, 24, seed=1)
+    with pytest.raises(ValueError):
+        oracle.gemm_epilogue_ex(p.A, p.B, None, None, 16, 8, 24, 1, 1.0, 0.0, W.FLAG_B_SYMMETRIC)
