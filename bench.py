@@ -466,25 +466,31 @@ def conv_row(ctx, device, peaks, flush):
 
 
 def symm_rows(ctx, device, peaks, flush):
-    """Symmetric A (CG_FLAG_A_SYMMETRIC) against the same call without the flag, on a memory-bound shape -- an
-    8192 x 8192 symmetric A (134 MB) times a 128-column B -- and on the compute-bound 4096-cube; + bias + SiLU.
-    Algorithmic bytes with the flag: the upper triangle of A (diagonal blocks whole), B, bias, D."""
+    """A symmetric operand (CG_FLAG_A_SYMMETRIC / CG_FLAG_B_SYMMETRIC) against the same call without the flag:
+    an 8192 x 8192 symmetric A (134 MB) times a 128-column B; the compute-bound 4096-cube with a symmetric A; and
+    128 rows of A against an 8192 x 8192 symmetric B (the skinny workload's shape); each + bias + SiLU.
+    Algorithmic bytes with the flag: the upper triangle of the symmetric operand (256-wide diagonal band whole),
+    the other operand, bias, D."""
     import torch
     out = {}
-    for m, n in ((8192, 128), (4096, 4096)):
+    for which, m, n, k in (("A", 8192, 128, 8192), ("A", 4096, 4096, 4096), ("B", 128, 8192, 8192)):
         g = torch.Generator(device=device)
         g.manual_seed(7)
-        a = torch.randn((m, m), device=device, generator=g)
-        a = (torch.triu(a) + torch.triu(a, 1).t()).to(torch.bfloat16).contiguous()
-        b = (torch.randn((n, m), device=device, generator=g) * (1.0 / 64.0)).to(torch.bfloat16)       # [N, K]
+        side = m if which == "A" else n
+        sym = torch.randn((side, side), device=device, generator=g) * (1.0 if which == "A" else 1.0 / 90.0)
+        sym = (torch.triu(sym) + torch.triu(sym, 1).t()).to(torch.bfloat16).contiguous()
+        if which == "A":
+            a, b = sym, (torch.randn((n, k), device=device, generator=g) * (1.0 / 64.0)).to(torch.bfloat16)       # B as [N, K]
+        else:
+            a, b = torch.randn((m, k), device=device, generator=g).to(torch.bfloat16), sym
         bias = torch.randn((n,), device=device, generator=g)
         d = torch.empty((m, n), device=device, dtype=torch.bfloat16)
         act = W.ACT_SILU | W.FLAG_B_COLMAJOR
         row = {}
-        for label, flag in (("symmetric", W.FLAG_A_SYMMETRIC), ("plain", 0)):
-            call = lambda: ctx.gemm_epilogue_ex(a, b, bias, None, d, m, n, m, 1, 1.0, 0.0, act | flag)
+        for label, flag in (("symmetric", W.FLAG_A_SYMMETRIC if which == "A" else W.FLAG_B_SYMMETRIC), ("plain", 0)):
+            call = lambda: ctx.gemm_epilogue_ex(a, b, bias, None, d, m, n, k, 1, 1.0, 0.0, act | flag)
             timed(call, 3, flush)
-            ts = timed(call, 10, flush)
+            ts = timed(call, 20, flush)
             ctx.check()
             row[f"{label}_us_best"] = min(ts) * 1e6
             row[f"{label}_us_median"] = float(np.median(ts)) * 1e6
@@ -492,17 +498,17 @@ def symm_rows(ctx, device, peaks, flush):
         lib = lambda: torch.matmul(a, b.t(), out=d)
         timed(lib, 3, flush)
         row["cublas_gemm_only_us_best"] = min(timed(lib, 10, flush)) * 1e6
-        flops = 2.0 * m * m * n
-        bytes_plain = 2.0 * (m * m + m * n + m * n) + 4.0 * n
-        bytes_symm = bytes_plain - 2.0 * (m * m - m * 256) / 2.0              # what lies below the 256-wide diagonal band is not read
+        flops = 2.0 * m * n * k
+        bytes_plain = 2.0 * (m * k + k * n + m * n) + 4.0 * n
+        bytes_symm = bytes_plain - 2.0 * (side * side - side * 256) / 2.0      # what lies below the 256-wide diagonal band is not read
         best = row["symmetric_us_best"] * 1e-6
-        row.update({"workload": f"symmetric A {m} x {m} bf16, B [{n}, {m}] (K-major), bias fp32, SiLU", "flops": flops,
+        row.update({"workload": f"symmetric {which}: M={m} N={n} K={k} bf16, B stored [N, K], bias fp32, SiLU", "flops": flops,
                     "algorithmic_bytes_plain": bytes_plain, "algorithmic_bytes_symmetric": bytes_symm,
                     "tflops_best": flops / best / 1e12, "gbs_best_of_symmetric_bytes": bytes_symm / best / 1e9,
                     "gbs_equivalent_of_plain_bytes": bytes_plain / best / 1e9,
                     "frac_hbm_of_measured": bytes_symm / best / 1e9 / peaks["hbm_gbs"],
                     "frac_tensor_of_measured_burst": flops / best / 1e12 / peaks["bf16_tflops"]})
-        out[f"{m}x{n}"] = row
+        out[f"{which}_{m}x{n}x{k}"] = row
     return out
 
 
@@ -539,7 +545,7 @@ def workload_table(ctx, device, peaks, names):
         out["next_tf32_8192"] = tf32_row(ctx, device, peaks, flush)
         out["next_diag_matmul_8192"] = diag_rows(ctx, device, peaks, flush)
         out["next_conv3x3_256"] = conv_row(ctx, device, peaks, flush)
-        out["next_symmetric_a"] = symm_rows(ctx, device, peaks, flush)
+        out["next_symmetric_operand"] = symm_rows(ctx, device, peaks, flush)
     return out
 
 

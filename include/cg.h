@@ -117,6 +117,13 @@ CG_API int cg_gemm_epilogue(cg_handle_t h, const void* A, const void* B, const v
  *                         inside the 256 x 256 squares on the diagonal; everything else there may hold anything.
  *                         bf16 operands only (with CG_FLAG_IN_F32: CG_ERR_UNSUPPORTED); tile shapes 128 x 128,
  *                         128 x 256 and the 256 x 256 pair tile (another forced shape: CG_ERR_INVALID_ARG)
+ *   CG_FLAG_B_SYMMETRIC   the same promise for B (N == K, else CG_ERR_INVALID_ARG; CG_FLAG_B_COLMAJOR is then
+ *                         immaterial: a symmetric matrix is its own transpose).  A k-block above a tile's diagonal
+ *                         block is fetched as stored rows k, columns n and multiplied as an N-major operand, every
+ *                         other block as rows n, columns k; nothing below the diagonal is read outside the
+ *                         256 x 256 squares on it.  This is the form that pays on a skinny problem (few rows of
+ *                         A against a large symmetric B): the traffic from DRAM halves.  Not together with
+ *                         CG_FLAG_A_SYMMETRIC or CG_FLAG_IN_F32 (CG_ERR_UNSUPPORTED); same tile shapes
  * and in *ex (NULL = all off, the call then equals cg_gemm_epilogue):
  *   row_scale, col_scale  device, fp32 [M] / [N], or NULL (= 1); they scale the product like alpha, never the bias;
  *                         shared by all batch entries
@@ -134,7 +141,7 @@ CG_API int cg_gemm_epilogue(cg_handle_t h, const void* A, const void* B, const v
  * unknown row_reduce code or a reduction without row_out.
  */
 enum { CG_FLAG_BIAS_PER_ROW = 1 << 10, CG_FLAG_B_BROADCAST = 1 << 11, CG_FLAG_CLAMP = 1 << 12, CG_FLAG_IN_F32 = 1 << 13,
-       CG_FLAG_A_SYMMETRIC = 1 << 14 };
+       CG_FLAG_A_SYMMETRIC = 1 << 14, CG_FLAG_B_SYMMETRIC = 1 << 15 };
 enum { CG_OUT_BF16 = 0, CG_OUT_F16 = 1, CG_OUT_F32 = 2 };
 enum { CG_REDUCE_NONE = 0, CG_REDUCE_SUM = 1, CG_REDUCE_MAX = 2, CG_REDUCE_LOGSUMEXP = 3 };
 typedef struct cg_epilogue_ex {

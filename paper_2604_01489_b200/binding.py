@@ -22,6 +22,7 @@ CG_FLAG_B_BROADCAST = 1 << 11
 CG_FLAG_CLAMP = 1 << 12
 CG_FLAG_IN_F32 = 1 << 13
 CG_FLAG_A_SYMMETRIC = 1 << 14
+CG_FLAG_B_SYMMETRIC = 1 << 15
 CG_OUT_BF16, CG_OUT_F16, CG_OUT_F32 = 0, 1, 2
 CG_REDUCE_NONE, CG_REDUCE_SUM, CG_REDUCE_MAX, CG_REDUCE_LOGSUMEXP = 0, 1, 2, 3
 

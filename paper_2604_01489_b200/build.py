@@ -10,7 +10,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcg.so")
 SOURCES = ["cg_api.cu", "cg_inst.cu"]
 HEADERS = ["cg_kernel.cuh", "cg_small.cuh", "cg_diag.cuh", "cg_reduce.cuh", "cg_instances.h", "cg_ptx.cuh", os.path.join("..", "..", "include", "cg.h")]
-INSTANCE_GROUPS = 8          # cg_inst.cu is compiled once per group of kernel instances, in parallel
+INSTANCE_GROUPS = 9          # cg_inst.cu is compiled once per group of kernel instances, in parallel
 OBJ_DIR = os.path.join(HERE, "build")
 
 

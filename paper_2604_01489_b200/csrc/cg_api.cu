@@ -153,6 +153,12 @@ bool lookup(int bn, int cgn, bool km, KernelEntry* out, int mode = MODE_GEMM) {
     if (cgn == 2 && bn == 512) { *out = entry<512, 2, true, MODE_CONV>(); return true; }
     return false;
   }
+  if (mode == MODE_SYMM_B) {  // symmetric B: the same three tile shapes; the matrix serves as its own K-major form
+    if (cgn == 1 && bn == 128) { *out = entry<128, 1, true, MODE_SYMM_B>(); return true; }
+    if (cgn == 1 && bn == 256) { *out = entry<256, 1, true, MODE_SYMM_B>(); return true; }
+    if (cgn == 2 && bn == 256) { *out = entry<256, 2, true, MODE_SYMM_B>(); return true; }
+    return false;
+  }
   if (mode == MODE_SYMM) {    // symmetric A: three tile shapes (see make_plan)
     if (cgn == 1 && bn == 128) { *out = km ? entry<128, 1, true, MODE_SYMM>() : entry<128, 1, false, MODE_SYMM>(); return true; }
     if (cgn == 1 && bn == 256) { *out = km ? entry<256, 1, true, MODE_SYMM>() : entry<256, 1, false, MODE_SYMM>(); return true; }
@@ -198,6 +204,9 @@ int prepare_kernels(cg_context* h) {
           CG_CUDA(h, cudaFuncSetAttribute(reinterpret_cast<const void*>(e.fn), cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           SMEM_LIMIT));
         if (lookup(bns[i], cgn, km != 0, &e, MODE_SYMM))
+          CG_CUDA(h, cudaFuncSetAttribute(reinterpret_cast<const void*>(e.fn), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          SMEM_LIMIT));
+        if (km != 0 && lookup(bns[i], cgn, true, &e, MODE_SYMM_B))
           CG_CUDA(h, cudaFuncSetAttribute(reinterpret_cast<const void*>(e.fn), cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           SMEM_LIMIT));
       }
@@ -299,7 +308,7 @@ int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, bool
       if (N >= 256 && tiles(BM, 256) >= sms) bn = 256;
     }
   }
-  if (mode == MODE_SYMM) {       // the symmetric form exists for 128- and 256-wide tiles and the 256 x 256 pair tile
+  if (mode == MODE_SYMM || mode == MODE_SYMM_B) {   // the symmetric forms exist for 128- and 256-wide tiles and the 256 x 256 pair tile
     if (cgn == 2 && bn == 128 && t.tile_n == 0) cgn = 1;
     if (bn == 64 && t.tile_n == 0) bn = 128;
     if (bn == 512 && t.tile_n == 0) bn = 256;
@@ -318,7 +327,10 @@ int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, bool
       return fail(h, CG_ERR_UNSUPPORTED, "cluster_split=%d does not fit tile_n=%d, K=%d", t.cluster_split, bn, K);
     csk = t.cluster_split;
   } else if (t.cluster_split == 0 && t.tile_n == 0 && t.num_units == 0 && cgn == 1) {
-    const int cand[3][2] = {{128, 2}, {256, 4}, {256, 2}};     // measured order on the skinny workload
+    // measured order on the skinny workload; with a symmetric B, whose DRAM traffic is halved, the 128-wide
+    // tile's MMA issue rate (an MMA costs 128 clocks whatever its N) is what is left, and the 256-wide tile wins
+    const int cand_gemm[3][2] = {{128, 2}, {256, 4}, {256, 2}}, cand_symm_b[3][2] = {{256, 4}, {128, 2}, {256, 2}};
+    const int (*cand)[2] = mode == MODE_SYMM_B ? cand_symm_b : cand_gemm;
     for (int i = 0; i < 3 && csk == 1; ++i) {
       const long long ctas = tiles(BM, cand[i][0]) * cand[i][1];
       if (csk_ok(cand[i][0], cand[i][1]) && ctas <= sms && ctas * 10 >= static_cast<long long>(sms) * 7) {
@@ -328,8 +340,9 @@ int make_plan(cg_context* h, int M, int N, int K, int batch, bool b_kmajor, bool
     }
   }
   KernelEntry e;
-  if (!lookup(bn, cgn, b_kmajor, &e, mode == MODE_SYMM ? MODE_SYMM : MODE_GEMM))
-    return fail(h, CG_ERR_INVALID_ARG, "no kernel for tile_n=%d cta_group=%d%s", bn, cgn, mode == MODE_SYMM ? " with a symmetric A" : "");
+  const bool symm_mode = mode == MODE_SYMM || mode == MODE_SYMM_B;
+  if (!lookup(bn, cgn, b_kmajor, &e, symm_mode ? mode : MODE_GEMM))
+    return fail(h, CG_ERR_INVALID_ARG, "no kernel for tile_n=%d cta_group=%d%s", bn, cgn, symm_mode ? " with a symmetric operand" : "");
 
   pl->bn = bn;
   pl->cg = cgn;
@@ -491,9 +504,10 @@ int host_pipelined(cg_context* h, const char* A, const char* B, const void* bias
 int launch(cg_context* h, const void* A, const void* B, const void* bias, const void* R, void* D, int M, int N, int K,
            int batch, float alpha, float beta, int act, cudaStream_t stream, const cg_epilogue_ex_t* ex = nullptr,
            const ConvGeom* conv = nullptr) {
-  const bool b_kmajor = (act & CG_FLAG_B_COLMAJOR) != 0;
-  const bool symm = (act & CG_FLAG_A_SYMMETRIC) != 0;
-  const bool ext_in_use = (act & (CG_FLAG_BIAS_PER_ROW | CG_FLAG_B_BROADCAST | CG_FLAG_CLAMP | CG_FLAG_IN_F32 | CG_FLAG_A_SYMMETRIC)) != 0 ||
+  const bool symm = (act & CG_FLAG_A_SYMMETRIC) != 0, symm_b = (act & CG_FLAG_B_SYMMETRIC) != 0;
+  const bool b_kmajor = (act & CG_FLAG_B_COLMAJOR) != 0 || symm_b;      // (a symmetric B is its own K-major form)
+  const bool ext_in_use = (act & (CG_FLAG_BIAS_PER_ROW | CG_FLAG_B_BROADCAST | CG_FLAG_CLAMP | CG_FLAG_IN_F32 | CG_FLAG_A_SYMMETRIC |
+                                  CG_FLAG_B_SYMMETRIC)) != 0 ||
                           (ex && (ex->row_scale || ex->col_scale || ex->out_dtype != CG_OUT_BF16 || ex->row_reduce));
   const int row_reduce = ex ? ex->row_reduce : 0;
   const bool store_d = D != nullptr;
@@ -508,7 +522,7 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   const bool tf32 = (act & CG_FLAG_IN_F32) != 0;
   const int bk_elems = tf32 ? BK / 2 : BK;
   const int in_dtype = tf32 ? CG_OUT_F32 : CG_OUT_BF16;           // (element type code of A and B)
-  const int mode = conv ? MODE_CONV : (symm ? MODE_SYMM : MODE_GEMM);
+  const int mode = conv ? MODE_CONV : (symm ? MODE_SYMM : (symm_b ? MODE_SYMM_B : MODE_GEMM));
   int rc = make_plan(h, M, N, K, batch, b_kmajor, beta != 0.0f, &pl, out_dtype == CG_OUT_F32 || !store_d, bk_elems, mode);
   if (rc != CG_OK) return rc;
   KernelEntry e;
@@ -521,6 +535,7 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   if (rc != CG_OK) return rc;
   const int b_entries = b_broadcast ? 1 : batch;
   if (conv) rc = make_map(h, &tmB, B, static_cast<uint64_t>(conv->KH) * conv->KW * conv->IC, N, 1, BK, e.sub_cols);
+  else if (symm_b) rc = make_map(h, &tmB, B, K, N, b_entries, 64, 64);   // serves blocks read as they are and mirrored ones
   else if (b_kmajor) rc = make_map(h, &tmB, B, K, N, b_entries, bk_elems, e.sub_cols, in_dtype);
   else rc = make_map(h, &tmB, B, N, K, b_entries, 64, BK);
   if (rc != CG_OK) return rc;
@@ -777,13 +792,17 @@ int cg_gemm_epilogue_ex(cg_handle_t h, const void* A, const void* B, const void*
     return fail(h, CG_ERR_INVALID_ARG, "row_reduce must be a CG_REDUCE_* code with a 4-byte aligned row_out");
   // with a row reduction D may be NULL (only the reduction is wanted)
   int rc = validate(h, A, B, bias, R, (!D && reducing) ? const_cast<void*>(A) : D, M, N, K, batch, beta, act,
-                    CG_FLAG_BIAS_PER_ROW | CG_FLAG_B_BROADCAST | CG_FLAG_CLAMP | CG_FLAG_IN_F32 | CG_FLAG_A_SYMMETRIC);
+                    CG_FLAG_BIAS_PER_ROW | CG_FLAG_B_BROADCAST | CG_FLAG_CLAMP | CG_FLAG_IN_F32 | CG_FLAG_A_SYMMETRIC |
+                        CG_FLAG_B_SYMMETRIC);
   if (rc != CG_OK) return rc;
   if ((act & CG_FLAG_IN_F32) && !(act & CG_FLAG_B_COLMAJOR))
     return fail(h, CG_ERR_UNSUPPORTED, "fp32 operands need B stored [batch,N,K] (CG_FLAG_B_COLMAJOR)");
   if ((act & CG_FLAG_A_SYMMETRIC) && M != K) return fail(h, CG_ERR_INVALID_ARG, "a symmetric A is square (got M=%d K=%d)", M, K);
-  if ((act & CG_FLAG_A_SYMMETRIC) && (act & CG_FLAG_IN_F32))
-    return fail(h, CG_ERR_UNSUPPORTED, "the symmetric form exists for bf16 operands only");
+  if ((act & CG_FLAG_B_SYMMETRIC) && N != K) return fail(h, CG_ERR_INVALID_ARG, "a symmetric B is square (got N=%d K=%d)", N, K);
+  if ((act & (CG_FLAG_A_SYMMETRIC | CG_FLAG_B_SYMMETRIC)) && (act & CG_FLAG_IN_F32))
+    return fail(h, CG_ERR_UNSUPPORTED, "the symmetric forms exist for bf16 operands only");
+  if ((act & CG_FLAG_A_SYMMETRIC) && (act & CG_FLAG_B_SYMMETRIC))
+    return fail(h, CG_ERR_UNSUPPORTED, "one symmetric operand per call");
   if ((rc = check_alignment(h, A, B, (act & CG_FLAG_BIAS_PER_ROW) ? nullptr : bias, R, D ? D : const_cast<void*>(A), beta, act)) != CG_OK)
     return rc;
   if (ex) {

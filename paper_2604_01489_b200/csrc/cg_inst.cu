@@ -3,7 +3,7 @@
 #include "cg_instances.h"
 
 #ifndef CG_INST_GROUP
-#error "compile with -DCG_INST_GROUP=<0..7>"
+#error "compile with -DCG_INST_GROUP=<0..8>"
 #endif
 
 namespace cg {
@@ -24,6 +24,8 @@ CG_INSTANCES_GROUP5(CG_DEFINE)
 CG_INSTANCES_GROUP6(CG_DEFINE)
 #elif CG_INST_GROUP == 7
 CG_INSTANCES_GROUP7(CG_DEFINE)
+#elif CG_INST_GROUP == 8
+CG_INSTANCES_GROUP8(CG_DEFINE)
 #else
 #error "CG_INST_GROUP out of range"
 #endif

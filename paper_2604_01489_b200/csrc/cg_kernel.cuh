@@ -34,7 +34,7 @@
 // MODE (template parameter) says what A is: a matrix (rank-3 map), an NHWC image read through rank-4
 // boxes (convolution as an implicit GEMM), or a square symmetric matrix of which only the blocks on or
 // above the diagonal are fetched (a block left of the diagonal comes from its mirror image and is
-// multiplied as an M-major operand).
+// multiplied as an M-major operand); or that B is such a symmetric matrix.
 //
 // With CG == 2 a pair of CTAs (cluster 2x1) shares one 256 x BN tile: each CTA loads its own
 // 128 rows of A and half of the B columns, the leader CTA issues tcgen05.mma.cta_group::2,
@@ -94,7 +94,7 @@ struct ConvGeom {
   int tiles_h, tiles_w;   // pixel tiles per image
 };
 constexpr int CONV_TILE_H = 8, CONV_TILE_W = 16;
-enum { MODE_GEMM = 0, MODE_CONV = 1, MODE_SYMM = 2 };    // what the A operand is (a template parameter of the kernel)
+enum { MODE_GEMM = 0, MODE_CONV = 1, MODE_SYMM = 2, MODE_SYMM_B = 3 };    // what the operands are (a template parameter of the kernel)
 
 struct KernelParams {
   int M, N, K, batch;
@@ -184,6 +184,7 @@ struct Cfg {
   static constexpr uint32_t IDESC = ptx::instr_desc_bf16(BM * CG, MMA_N, !B_KMAJOR);
   static constexpr uint32_t IDESC_TF32 = ptx::instr_desc_tf32(BM * CG, MMA_N);
   static constexpr uint32_t IDESC_A_MIRRORED = IDESC | ptx::INSTR_DESC_A_MN_MAJOR;   // A read M-major (symmetric A, mirrored block)
+  static constexpr uint32_t IDESC_B_MIRRORED = IDESC | ptx::INSTR_DESC_B_MN_MAJOR;   // B read N-major (symmetric B, mirrored block)
   __host__ __device__ static constexpr int layout_bytes(int stages, bool with_r) {
     return stages * STAGE_BYTES + FIXED_BYTES + (with_r ? R_BYTES : 0);
   }
@@ -456,6 +457,8 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
   using C = Cfg<BN, CG, B_KMAJOR>;
   constexpr bool CONV = (MODE == MODE_CONV);     // A is an NHWC image read through rank-4 boxes
   constexpr bool SYMM = (MODE == MODE_SYMM);     // A is square and symmetric: only blocks on or above the diagonal are read
+  constexpr bool SYMM_B = (MODE == MODE_SYMM_B); // the same for B (instantiated with B_KMAJOR: a symmetric matrix is both)
+  static_assert(!SYMM_B || B_KMAJOR, "the symmetric-B form takes the K-major instance");
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = ptx::smem_u32(smem_raw);
   const uint32_t pad = ((raw_addr + 1023u) & ~1023u) - raw_addr;
@@ -516,7 +519,17 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     for (int h = 0; h < C::NSUB; ++h) {
       const int nh = n0 + h * C::MMA_N;
       const uint32_t dst = b_dst + h * C::SUB_B_BYTES;
-      if constexpr (B_KMAJOR) {
+      if constexpr (SYMM_B) {
+        // Symmetric B through 64 x 64 boxes.  A k-block above the tile's diagonal block (k < n) is fetched as
+        // rows k, columns n -- above the diagonal -- and lands N-major like a row-major B; every other block is
+        // fetched as rows n, columns k, the K-major form.
+        const bool mirrored = k0 + BK <= n0;
+#pragma unroll
+        for (int j = 0; j < C::SUB_COLS / 64; ++j) {
+          if (mirrored) ptx::tma_load_3d(dst + j * (64 * BK * 2), &tmB, bar, nh + j * 64, k0, bb);
+          else ptx::tma_load_3d(dst + j * (64 * BK * 2), &tmB, bar, k0, nh + j * 64, bb);
+        }
+      } else if constexpr (B_KMAJOR) {
         ptx::tma_load_3d(dst, &tmB, bar, k0, nh, bb);
       } else {
 #pragma unroll
@@ -612,7 +625,14 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             for (int h = 0; h < C::NSUB; ++h) {
               const int nh = n0 + h * C::MMA_N;
               const uint32_t dst = b_dst + h * C::SUB_B_BYTES;
-              if constexpr (B_KMAJOR) {
+              if constexpr (SYMM_B) {
+                const bool mirrored = k0 + BK <= nt * BN;           // one decision for the pair
+#pragma unroll
+                for (int j = 0; j < C::SUB_COLS / 64; ++j) {
+                  if (mirrored) ptx::tma_load_3d_pair(dst + j * (64 * BK * 2), &tmB, bar, nh + j * 64, k0, bb);
+                  else ptx::tma_load_3d_pair(dst + j * (64 * BK * 2), &tmB, bar, k0, nh + j * 64, bb);
+                }
+              } else if constexpr (B_KMAJOR) {
                 ptx::tma_load_3d_pair(dst, &tmB, bar, k0, nh, bb);
               } else {
 #pragma unroll
@@ -690,17 +710,21 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
       // symmetric A: a mirrored k-block is an M-major operand (same form as a row-major B block)
       const uint32_t a_lo0_mirrored = static_cast<uint32_t>(ptx::smem_desc_sw128(ring_addr, 64 * BK * 2, 8 * 128));
       constexpr uint32_t A_KSTEP_MIRRORED = (UMMA_K * 128) >> 4;         // +16 k-rows
+      // symmetric B: a mirrored k-block is N-major (what a row-major B block always is)
+      const uint32_t b_lo0_mirrored = static_cast<uint32_t>(ptx::smem_desc_sw128(ring_addr + C::A_BYTES, 64 * BK * 2, 8 * 128));
+      constexpr uint32_t B_KSTEP_MIRRORED = (UMMA_K * 128) >> 4;
       auto desc = [&](uint32_t lo) -> uint64_t { return (static_cast<uint64_t>(desc_hi) << 32) | lo; };
       while (ok && wi.next(s)) {
         if (!wait_bar(ptx::smem_u32(&ctrl->acc_empty[acc]), acc_phase ^ 1u, ctrl, p)) { ok = false; break; }
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
         uint32_t accumulate = 0;
-        int tile_row0 = 0;                       // symmetric A: first row of this (pair) tile
-        if constexpr (SYMM) {
+        int tile_row0 = 0, tile_col0 = 0;        // symmetric A / B: first row / column of this (pair) tile
+        if constexpr (SYMM || SYMM_B) {
           int tb, tmt, tnt;
           decode_tile(p, s.tile, tb, tmt, tnt);
           tile_row0 = tmt * (BM * CG);
+          tile_col0 = tnt * BN;
         }
         for (int kb = s.kb0; kb < s.kb1; ++kb) {
           if (!wait_bar(full0 + stage * 8, phase, ctrl, p)) { ok = false; break; }
@@ -709,20 +733,22 @@ gemm_epilogue_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
           const bool mirrored = SYMM && (kb + 1) * BK <= tile_row0;
           const uint32_t a_lo = (mirrored ? a_lo0_mirrored : a_lo0) + stage * STAGE_STEP;
           const uint32_t a_kstep = mirrored ? A_KSTEP_MIRRORED : A_KSTEP;
-          const uint32_t idesc = mirrored ? C::IDESC_A_MIRRORED : C::IDESC;
-          const uint32_t b_lo = b_lo0 + stage * STAGE_STEP;
+          const bool mirrored_b = SYMM_B && (kb + 1) * BK <= tile_col0;
+          const uint32_t idesc = mirrored ? C::IDESC_A_MIRRORED : (mirrored_b ? C::IDESC_B_MIRRORED : C::IDESC);
+          const uint32_t b_lo = (mirrored_b ? b_lo0_mirrored : b_lo0) + stage * STAGE_STEP;
+          const uint32_t b_kstep = mirrored_b ? B_KSTEP_MIRRORED : B_KSTEP;
           if (kb != last_kb || tail_nk == BK / UMMA_K) {
 #pragma unroll
             for (int k = 0; k < BK / UMMA_K; ++k)
 #pragma unroll
               for (int h = 0; h < C::NSUB; ++h)
-                mma(d_tmem + h * C::MMA_N, desc(a_lo + k * a_kstep), desc(b_lo + k * B_KSTEP + h * SUB_STEP),
+                mma(d_tmem + h * C::MMA_N, desc(a_lo + k * a_kstep), desc(b_lo + k * b_kstep + h * SUB_STEP),
                     k == 0 ? accumulate : 1u, idesc);
           } else {
             for (int k = 0; k < tail_nk; ++k)     // K tail: skip 16-wide steps that are all padding
 #pragma unroll
               for (int h = 0; h < C::NSUB; ++h)
-                mma(d_tmem + h * C::MMA_N, desc(a_lo + k * a_kstep), desc(b_lo + k * B_KSTEP + h * SUB_STEP),
+                mma(d_tmem + h * C::MMA_N, desc(a_lo + k * a_kstep), desc(b_lo + k * b_kstep + h * SUB_STEP),
                     (k > 0) ? 1u : accumulate, idesc);
           }
           accumulate = 1u;

@@ -277,6 +277,7 @@ __host__ __device__ constexpr uint32_t instr_desc_bf16(int m, int n, bool b_mn_m
 }
 
 constexpr uint32_t INSTR_DESC_A_MN_MAJOR = 1u << 15;     // A operand stored M-major ("transposed") instead of K-major
+constexpr uint32_t INSTR_DESC_B_MN_MAJOR = 1u << 16;     // B operand stored N-major
 
 // Instruction descriptor, kind::tf32: as above with TF32 A and B (format code 2), both K-major.
 __host__ __device__ constexpr uint32_t instr_desc_tf32(int m, int n) {

@@ -130,7 +130,7 @@ def test_error_codes(ctx):
     call = lambda act=0, **ex: cg.cg_gemm_epilogue_ex(h, dev["A"], dev["B"], None, None, dev["D"], 64, 64, 64, 1, 1.0, 0.0, act, **ex)
     assert call(act=cg.CG_FLAG_CLAMP, clamp_lo=1.0, clamp_hi=-1.0) == cg.CG_ERR_INVALID_ARG
     assert call(out_dtype=3) == cg.CG_ERR_INVALID_ARG and call(out_dtype=-1) == cg.CG_ERR_INVALID_ARG
-    assert call(act=1 << 15) == cg.CG_ERR_INVALID_ARG
+    assert call(act=1 << 16) == cg.CG_ERR_INVALID_ARG
     assert call(row_scale=dev["A"].data_ptr() + 2) == cg.CG_ERR_UNSUPPORTED
     # the base entry point does not know the extended flags
     assert cg.cg_gemm_epilogue(h, dev["A"], dev["B"], None, None, dev["D"], 64, 64, 64, 1, 1.0, 0.0, cg.CG_FLAG_CLAMP) == cg.CG_ERR_INVALID_ARG

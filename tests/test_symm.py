@@ -1,5 +1,5 @@
-"""GPU parity of the symmetric-A form (CG_FLAG_A_SYMMETRIC) against the CPU oracle.  The oracle takes the upper
-triangle as the matrix; the kernel gets a symmetric A in which everything it promises not to read -- below the
+"""GPU parity of the symmetric forms (CG_FLAG_A_SYMMETRIC, CG_FLAG_B_SYMMETRIC) against the CPU oracle.  The oracle takes the upper
+triangle as the matrix; the kernel gets a symmetric operand in which everything it promises not to read -- below the
 diagonal, outside the 256 x 256 squares on it -- is a NaN, so a single stray read fails the comparison.
 Integer-valued operands with a linear epilogue must match bit for bit; the rest within the bf16 tolerance
 |D_gpu - D_ref| <= 1e-2 (|D_ref| + 1), relative Frobenius error <= 5e-3."""
@@ -29,6 +29,8 @@ def ctx():
 
 
 def poisoned(p):
+    if p.act & W.FLAG_B_SYMMETRIC:
+        return dataclasses.replace(p, B=W.poison_below_blocks(p.B, 256))
     return dataclasses.replace(p, A=W.poison_below_blocks(p.A, 256))
 
 
@@ -124,4 +126,61 @@ def test_error_codes(ctx):
     ctx.set_tuning(tile_n=512, cta_group=2)
     assert call() == cg.CG_ERR_INVALID_ARG                                            # no symmetric form of that tile
     ctx.set_tuning(reset=True)
+    ctx.check()
+
+
+# ---------------------------------------------------------------- symmetric B
+
+SIZES_B = [(72, 136, 1), (264, 520, 2), (136, 904, 1), (512, 1024, 1)]       # (M, N = K, batch)
+
+
+@pytest.mark.parametrize("colmajor", [False, True], ids=["Brow", "Bcol"])
+@pytest.mark.parametrize("plan", PLANS, ids=lambda d: "auto" if not d else f"bn{d['tile_n']}cg{d['cta_group']}")
+@pytest.mark.parametrize("size", SIZES_B, ids=lambda s: "x".join(map(str, s)))
+def test_symmetric_b_integer_operands_bit_exact(ctx, oracle, size, plan, colmajor):
+    m, n, batch = size
+    act = W.ACT_RELU | W.FLAG_B_SYMMETRIC | (W.FLAG_B_COLMAJOR if colmajor else 0)
+    p = W.make(m, n, n, batch, seed=m + n, act=act, alpha=1.0, beta=1.0, A=SI, B=SI, bias=SI, R=SI)
+    pl = check(ctx, oracle, p, exact=True, **plan)
+    assert pl["latency_kernel"] == 0
+
+
+@pytest.mark.parametrize("plan", PLANS, ids=lambda d: "auto" if not d else f"bn{d['tile_n']}cg{d['cta_group']}")
+def test_symmetric_b_normal_operands_with_activation(ctx, oracle, plan):
+    p = W.make(392, 776, 776, 2, seed=15, act=W.ACT_GELU_TANH | W.FLAG_B_SYMMETRIC | W.FLAG_B_BROADCAST, A=("normal", 1.0),
+               B=("normal", 0.05), bias=("normal", 0.5))
+    check(ctx, oracle, p, **plan)
+
+
+@pytest.mark.parametrize("tuning", [dict(tile_n=128, cluster_split=2), dict(tile_n=256, cluster_split=4),
+                                    dict(tile_n=128, cta_group=1, num_units=24, dp_units=0),
+                                    dict(tile_n=256, cta_group=2, num_units=7, dp_units=2)],
+                         ids=["cluster2", "cluster4", "splitk", "streamk-pairs"])
+def test_symmetric_b_split_plans(ctx, oracle, tuning):
+    p = W.make(256, 1024, 1024, 1, seed=16, act=W.ACT_NONE | W.FLAG_B_SYMMETRIC, alpha=0.5, A=SI, B=SI)
+    check(ctx, oracle, p, exact=True, **tuning)
+
+
+def test_symmetric_b_skinny_memory_bound_shape_sampled_rows(ctx, oracle):
+    """The shape the flag pays on: few rows of A against a large symmetric B."""
+    m, n = 128, 4096
+    p = W.make(m, n, n, 1, seed=17, act=W.ACT_SILU | W.FLAG_B_SYMMETRIC, A=("normal", 1.0), B=("normal", 1.0 / 64.0),
+               bias=("normal", 0.1))
+    rows = np.array([0, 1, 31, 32, 63, 64, 100, 127], dtype=np.int64)
+    pl = check(ctx, oracle, p, rows=rows)
+    assert pl["num_units"] > pl["num_tiles"]            # K is split
+
+
+def test_symmetric_b_error_codes(ctx):
+    import paper_2604_01489_b200 as cg
+    p = W.make(64, 128, 128, seed=1)
+    dev = PU.to_device(p)
+    h = ctx.handle
+    ctx.set_tuning(reset=True)
+    call = lambda N=128, K=128, act=cg.CG_FLAG_B_SYMMETRIC: cg.cg_gemm_epilogue_ex(h, dev["A"], dev["B"], None, None, dev["D"], 64, N, K,
+                                                                                 1, 1.0, 0.0, act)
+    assert call() == cg.CG_OK
+    assert call(N=64) == cg.CG_ERR_INVALID_ARG                                        # not square
+    assert call(act=cg.CG_FLAG_B_SYMMETRIC | cg.CG_FLAG_IN_F32 | cg.CG_FLAG_B_COLMAJOR) == cg.CG_ERR_UNSUPPORTED
+    assert call(act=cg.CG_FLAG_B_SYMMETRIC | cg.CG_FLAG_A_SYMMETRIC) == cg.CG_ERR_INVALID_ARG     # (64 x 128 A is not square)
     ctx.check()
