@@ -616,7 +616,7 @@ int launch(cg_context* h, const void* A, const void* B, const void* bias, const 
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = (attr[0].val.clusterDim.x > 1 || getenv("CG_ALWAYS_CLUSTER")) ? 1 : 0;      // a plain launch when there is no cluster
+  cfg.numAttrs = attr[0].val.clusterDim.x > 1 ? 1 : 0;      // a plain launch when there is no cluster
   void* args[5] = {&tmA, &tmB, &tmD, &tmR, &p};
   CG_CUDA(h, cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(e.fn), args));
   if (row_reduce) {
